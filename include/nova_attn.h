@@ -1,0 +1,114 @@
+/*
+ * nova_attn.h - C ABI of libnova_attn: fused causal multi-head attention for NVIDIA B200 (sm_100a).
+ *
+ * The library implements, as hand-written CUDA, the attention sub-graph that the Nova compiler
+ * collapses into single kernels (paper Section 4.2, "Attention as a First-Class Lowering"):
+ *   forward  - scores = scale * Q K^T, causal mask from indices, online base-2 softmax, O = P V,
+ *              log-sum-exp of every row saved for the backward pass;
+ *   backward - P recomputed from the saved log-sum-exp (never stored), dV, dP, dS, dQ, dK.
+ *
+ * Conventions shared by every entry point
+ *   - All tensor pointers are DEVICE pointers on the current CUDA device, owned by the caller, and
+ *     must be 16-byte aligned, non-overlapping, and stay valid until the work enqueued on `stream`
+ *     has finished.  Inputs are never modified; outputs are fully overwritten.
+ *   - Q, K, V, O, dO, dQ, dK, dV: bf16, shape [B, H, T, D], contiguous (D fastest).
+ *     LSE, Delta: fp32, shape [B, H, T].
+ *   - D must be 64 or 128.  Any T >= 1 is accepted (partial tiles are handled inside).  Self
+ *     attention only (queries and keys share T); no dropout, bias or grouped heads.
+ *   - `scale` multiplies Q K^T before the softmax and must be finite and > 0.
+ *   - `causal` != 0 keeps key j for query i iff j <= i; 0 keeps every key.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Calls only
+ *     enqueue work on that stream: they never synchronise the device and never allocate device
+ *     memory.
+ *   - Return value: NOVA_ATTN_OK (0) or a negative nova_attn_status.  Arguments are validated on the
+ *     host before anything is launched; a failed call has launched nothing.
+ *   - Every wait inside the kernels is bounded.  If one expires (which indicates a bug or a broken
+ *     device, never a property of the input) the kernel records NOVA_ATTN_ERR_TIMEOUT in a device
+ *     status word, releases what it holds and returns; nova_attn_poll_device_status() reads the word.
+ */
+#ifndef NOVA_ATTN_H_
+#define NOVA_ATTN_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum nova_attn_status {
+    NOVA_ATTN_OK = 0,
+    NOVA_ATTN_ERR_NULL = -1,        /* a required pointer is NULL */
+    NOVA_ATTN_ERR_SHAPE = -2,       /* B, H or T <= 0, or B*H*T*D overflows the supported range */
+    NOVA_ATTN_ERR_UNSUPPORTED = -3, /* D not in {64, 128}, or the device is not sm_100 */
+    NOVA_ATTN_ERR_ALIGNMENT = -4,   /* a tensor pointer is not 16-byte aligned */
+    NOVA_ATTN_ERR_SCALE = -5,       /* scale is not finite or not > 0 */
+    NOVA_ATTN_ERR_WORKSPACE = -6,   /* workspace is NULL or smaller than nova_attn_bwd_workspace_bytes */
+    NOVA_ATTN_ERR_CUDA = -7,        /* a CUDA runtime/driver call failed; see nova_attn_last_cuda_error */
+    NOVA_ATTN_ERR_TIMEOUT = -8      /* a bounded device-side wait expired (reported by the poll call) */
+} nova_attn_status;
+
+/*
+ * Forward pass (paper Section 4.2: the nova.online_attention loop - score contraction, index mask,
+ * running max / sum in base 2, value contraction, causal loop clamp, 1/sum in the epilogue, and
+ * "saves the log-sum-exp of each row for the backward pass").
+ *   Q, K, V : in,  bf16 [B,H,T,D]
+ *   O       : out, bf16 [B,H,T,D]   O_i = sum_j softmax_j(scale * q_i.k_j) v_j over the kept keys
+ *   LSE     : out, fp32 [B,H,T]     natural-log log-sum-exp of the kept scaled scores of row i
+ * bf16 operands feed the tensor cores, accumulation and all softmax arithmetic are fp32 (Section 4.3).
+ */
+int nova_attn_fwd(const void* Q, const void* K, const void* V, void* O, float* LSE,
+                  int B, int H, int T, int D, float scale, int causal, void* stream);
+
+/*
+ * Backward preprocess: Delta_i = sum_d dO[i,d] * O[i,d], the row term of the softmax Jacobian
+ * (equal to sum_j P_ij dP_ij).  The paper's backward (Section 4.2, "The Backward Pass") does not
+ * spell this step out; it is the standard way to obtain dS = P * (dP - Delta) without a second
+ * reduction over keys.  Memory bound: reads O and dO once.
+ *   O, dO : in,  bf16 [B,H,T,D]   (O as written by nova_attn_fwd)
+ *   Delta : out, fp32 [B,H,T]
+ */
+int nova_attn_bwd_preprocess(const void* O, const void* dO, float* Delta,
+                             int B, int H, int T, int D, void* stream);
+
+/*
+ * Bytes of scratch nova_attn_bwd needs: an fp32 accumulator for dQ, [B,H,T,D].
+ * Returns 0 if the shape is invalid.
+ */
+size_t nova_attn_bwd_workspace_bytes(int B, int H, int T, int D);
+
+/*
+ * Backward pass (paper Section 4.2, "The Backward Pass": dQ reduces over keys, dK and dV reduce over
+ * queries, the probability matrix is recomputed from the cached log-sum-exp and never stored; the
+ * causal loop bound is raised so tiles above the diagonal are never visited).
+ *   Q, K, V, dO : in, bf16 [B,H,T,D]
+ *   O           : in, bf16 [B,H,T,D]; accepted for symmetry and ignored (Delta already carries it)
+ *   LSE, Delta  : in, fp32 [B,H,T] from nova_attn_fwd / nova_attn_bwd_preprocess
+ *   dQ, dK, dV  : out, bf16 [B,H,T,D]; gradient of sum(O * dO) with respect to Q, K, V
+ *   workspace   : device scratch of at least nova_attn_bwd_workspace_bytes(B,H,T,D) bytes, 16-byte
+ *                 aligned; zeroed by the call itself on `stream`; contents afterwards unspecified.
+ * dQ is accumulated in fp32 across key tiles with floating-point atomics, so its low-order bits may
+ * differ from run to run; dK and dV are deterministic.
+ */
+int nova_attn_bwd(const void* Q, const void* K, const void* V, const void* O, const void* dO,
+                  const float* LSE, const float* Delta, void* dQ, void* dK, void* dV,
+                  int B, int H, int T, int D, float scale, int causal,
+                  void* workspace, size_t workspace_bytes, void* stream);
+
+/* Static, never-freed description of a status code. */
+const char* nova_attn_status_string(int status);
+
+/* CUDA error code (cudaError_t or CUresult, as int) behind the calling thread's last
+ * NOVA_ATTN_ERR_CUDA; 0 if none. */
+int nova_attn_last_cuda_error(void);
+
+/*
+ * Synchronises `stream`, then reads and clears the device status word of the current device.
+ * Returns NOVA_ATTN_OK, NOVA_ATTN_ERR_TIMEOUT (a kernel gave up on a bounded wait; its outputs are
+ * invalid) or NOVA_ATTN_ERR_CUDA.
+ */
+int nova_attn_poll_device_status(void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* NOVA_ATTN_H_ */

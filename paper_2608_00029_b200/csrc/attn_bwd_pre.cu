@@ -1,0 +1,107 @@
+// Memory-bound helpers of the backward pass.
+//   bwd_preprocess_kernel: Delta_i = sum_d dO[i,d] * O[i,d]   (row term of the softmax Jacobian)
+//   dq_convert_kernel:     dQ = bf16(scale * fp32 accumulator)
+// Both stream their inputs once with 16-byte loads; rows are split over D/8 lanes and reduced with
+// xor-shuffles.  Grids are sized in multiples of the SM count.
+#include "kernels.h"
+#include "ptx.cuh"
+
+namespace nova {
+namespace {
+
+__device__ __forceinline__ float dot8_bf16(const uint4& a, const uint4& b) {
+    const __nv_bfloat162* pa = reinterpret_cast<const __nv_bfloat162*>(&a);
+    const __nv_bfloat162* pb = reinterpret_cast<const __nv_bfloat162*>(&b);
+    float acc = 0.f;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float2 fa = __bfloat1622float2(pa[i]);
+        const float2 fb = __bfloat1622float2(pb[i]);
+        acc = fmaf(fa.x, fb.x, acc);
+        acc = fmaf(fa.y, fb.y, acc);
+    }
+    return acc;
+}
+
+// LPR = lanes per row = D/8 (8 for D=64, 16 for D=128); each lane owns 8 consecutive bf16.
+template <int LPR, int UNROLL>
+__global__ void __launch_bounds__(256) bwd_preprocess_kernel(const uint4* __restrict__ O, const uint4* __restrict__ dO,
+                                                             float* __restrict__ Delta, long long rows) {
+    const long long tid = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+    const long long nthreads = static_cast<long long>(gridDim.x) * blockDim.x;
+    const long long rows_per_pass = nthreads / LPR;
+    const int sub = static_cast<int>(tid % LPR);
+    long long r = tid / LPR;
+    for (; r < rows; r += rows_per_pass * UNROLL) {
+        uint4 a[UNROLL], b[UNROLL];
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+            const long long ru = r + u * rows_per_pass;
+            if (ru < rows) {
+                a[u] = __ldg(O + ru * LPR + sub);
+                b[u] = __ldg(dO + ru * LPR + sub);
+            } else {
+                a[u] = make_uint4(0, 0, 0, 0);
+                b[u] = make_uint4(0, 0, 0, 0);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+            float acc = dot8_bf16(a[u], b[u]);
+#pragma unroll
+            for (int off = LPR / 2; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+            const long long ru = r + u * rows_per_pass;
+            if (sub == 0 && ru < rows) Delta[ru] = acc;
+        }
+    }
+}
+
+__global__ void __launch_bounds__(256) dq_convert_kernel(const float4* __restrict__ acc, uint4* __restrict__ dQ,
+                                                         long long n8, float scale) {
+    const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
+    for (long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; i < n8; i += stride) {
+        const float4 a = __ldcs(acc + 2 * i);
+        const float4 b = __ldcs(acc + 2 * i + 1);
+        uint4 v;
+        v.x = pack_bf16x2(a.x * scale, a.y * scale);
+        v.y = pack_bf16x2(a.z * scale, a.w * scale);
+        v.z = pack_bf16x2(b.x * scale, b.y * scale);
+        v.w = pack_bf16x2(b.z * scale, b.w * scale);
+        dQ[i] = v;
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_attn_bwd_preprocess(const __nv_bfloat16* O, const __nv_bfloat16* dO, float* Delta,
+                                       long long rows, int D, int num_sms, cudaStream_t stream) {
+    constexpr int kThreads = 256, kUnroll = 4;
+    const int lpr = D / 8;
+    const long long rows_per_block = kThreads / lpr * kUnroll;
+    long long blocks = (rows + rows_per_block - 1) / rows_per_block;
+    const long long cap = static_cast<long long>(num_sms) * 8;
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    const uint4* o4 = reinterpret_cast<const uint4*>(O);
+    const uint4* d4 = reinterpret_cast<const uint4*>(dO);
+    if (D == 64)
+        bwd_preprocess_kernel<8, kUnroll><<<static_cast<unsigned>(blocks), kThreads, 0, stream>>>(o4, d4, Delta, rows);
+    else
+        bwd_preprocess_kernel<16, kUnroll><<<static_cast<unsigned>(blocks), kThreads, 0, stream>>>(o4, d4, Delta, rows);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_dq_convert(const float* dq_acc, __nv_bfloat16* dQ, long long n, float scale, int num_sms,
+                              cudaStream_t stream) {
+    constexpr int kThreads = 256;
+    const long long n8 = n / 8;  // D is a multiple of 8, so n is too
+    long long blocks = (n8 + kThreads - 1) / kThreads;
+    const long long cap = static_cast<long long>(num_sms) * 8;
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    dq_convert_kernel<<<static_cast<unsigned>(blocks), kThreads, 0, stream>>>(
+        reinterpret_cast<const float4*>(dq_acc), reinterpret_cast<uint4*>(dQ), n8, scale);
+    return cudaGetLastError();
+}
+
+}  // namespace nova

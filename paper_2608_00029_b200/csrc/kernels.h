@@ -1,0 +1,43 @@
+// Internal launch interface between the C ABI (api.cu) and the kernels.  Not installed.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace nova {
+
+constexpr int kBlockQ = 128;        // query rows per tile (UMMA M)
+constexpr int kBlockK = 128;        // keys per tile
+constexpr int kBoxCols = 64;        // bf16 elements per 128-byte swizzled row (TMA box inner extent)
+constexpr int kHalfTileBytes = 128 * 128;  // one [128 rows x 64 bf16] box
+
+struct AttnShape {
+    int B, H, T, D;
+    int causal;
+    float scale;
+};
+
+// Forward: tensor maps are 3-D [D, T, B*H] bf16 with a [64, 128, 1] box and 128-byte swizzle.
+cudaError_t launch_attn_fwd(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV,
+                            __nv_bfloat16* O, float* LSE, const AttnShape& s, int* dev_status,
+                            cudaStream_t stream);
+cudaError_t configure_attn_fwd();
+
+cudaError_t launch_attn_bwd_preprocess(const __nv_bfloat16* O, const __nv_bfloat16* dO, float* Delta,
+                                       long long rows, int D, int num_sms, cudaStream_t stream);
+
+// Backward main kernel: accumulates unscaled dQ into `dq_acc` (fp32 [B,H,T,D], zeroed beforehand),
+// writes dK and dV.
+cudaError_t launch_attn_bwd(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV,
+                            const CUtensorMap& tmdO, const float* LSE, const float* Delta, float* dq_acc,
+                            __nv_bfloat16* dK, __nv_bfloat16* dV, const AttnShape& s, int* dev_status,
+                            cudaStream_t stream);
+cudaError_t configure_attn_bwd();
+
+// dQ = bf16(scale * dq_acc)
+cudaError_t launch_dq_convert(const float* dq_acc, __nv_bfloat16* dQ, long long n, float scale, int num_sms,
+                              cudaStream_t stream);
+
+}  // namespace nova

@@ -1,0 +1,144 @@
+"""ctypes binding of libnova_attn.so: same names as the C ABI, argument marshalling only.
+
+Every step of the attention path runs inside the CUDA library; PyTorch is used here for device
+memory and streams.  There is no CPU fallback: if the shared library is missing or a call fails, an
+exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libnova_attn.so")
+_lib = None
+
+OK = 0
+ERR_NULL, ERR_SHAPE, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_SCALE, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(-1, -9, -1)
+
+
+class NovaAttnError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        lib = load()
+        msg = lib.nova_attn_status_string(status).decode()
+        extra = f" (cuda error {lib.nova_attn_last_cuda_error()})" if status == ERR_CUDA else ""
+        super().__init__(f"{where}: {msg}{extra} [status {status}]")
+
+
+def load():
+    """Load the shared library (once).  Raises if it has not been built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            f"{LIB_PATH} not found: build it with `python -m paper_2608_00029_b200.build` "
+            "(there is no CPU fallback for this library)")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, fp, i, f, sz = ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
+    lib.nova_attn_fwd.argtypes = [vp, vp, vp, vp, fp, i, i, i, i, f, i, vp]
+    lib.nova_attn_fwd.restype = i
+    lib.nova_attn_bwd_preprocess.argtypes = [vp, vp, fp, i, i, i, i, vp]
+    lib.nova_attn_bwd_preprocess.restype = i
+    lib.nova_attn_bwd_workspace_bytes.argtypes = [i, i, i, i]
+    lib.nova_attn_bwd_workspace_bytes.restype = sz
+    lib.nova_attn_bwd.argtypes = [vp] * 5 + [fp, fp, vp, vp, vp, i, i, i, i, f, i, vp, sz, vp]
+    lib.nova_attn_bwd.restype = i
+    lib.nova_attn_status_string.argtypes = [i]
+    lib.nova_attn_status_string.restype = ctypes.c_char_p
+    lib.nova_attn_last_cuda_error.argtypes = []
+    lib.nova_attn_last_cuda_error.restype = i
+    lib.nova_attn_poll_device_status.argtypes = [vp]
+    lib.nova_attn_poll_device_status.restype = i
+    if hasattr(lib, "nova_attn_bwd_static_scratch"):
+        lib.nova_attn_bwd_static_scratch.argtypes = [vp] * 5 + [fp, fp, vp, vp, vp, i, i, i, i, f, i, vp]
+        lib.nova_attn_bwd_static_scratch.restype = i
+        lib.nova_attn_static_scratch_bytes.argtypes = []
+        lib.nova_attn_static_scratch_bytes.restype = sz
+    _lib = lib
+    return lib
+
+
+def _stream_ptr(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return int(stream.cuda_stream)
+
+
+def _ptr(t) -> int:
+    return 0 if t is None else int(t.data_ptr())
+
+
+def _check_bf16(name, t, shape=None):
+    if t.dtype != torch.bfloat16 or not t.is_cuda or not t.is_contiguous():
+        raise TypeError(f"{name} must be a contiguous CUDA bf16 tensor")
+    if shape is not None and tuple(t.shape) != tuple(shape):
+        raise ValueError(f"{name} has shape {tuple(t.shape)}, expected {tuple(shape)}")
+
+
+def _check_f32(name, t, shape):
+    if t.dtype != torch.float32 or not t.is_cuda or not t.is_contiguous() or tuple(t.shape) != tuple(shape):
+        raise TypeError(f"{name} must be a contiguous CUDA fp32 tensor of shape {tuple(shape)}")
+
+
+def nova_attn_status_string(status: int) -> str:
+    return load().nova_attn_status_string(int(status)).decode()
+
+
+def nova_attn_bwd_workspace_bytes(B: int, H: int, T: int, D: int) -> int:
+    return int(load().nova_attn_bwd_workspace_bytes(B, H, T, D))
+
+
+def nova_attn_fwd(Q, K, V, O, LSE, scale: float, causal: bool = True, stream=None) -> None:
+    """O, LSE <- attention(Q, K, V); tensors are [B,H,T,D] bf16, LSE [B,H,T] fp32, all preallocated."""
+    _check_bf16("Q", Q)
+    B, H, T, D = Q.shape
+    for n, t in (("K", K), ("V", V), ("O", O)):
+        _check_bf16(n, t, Q.shape)
+    _check_f32("LSE", LSE, (B, H, T))
+    rc = load().nova_attn_fwd(_ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(LSE), B, H, T, D, float(scale),
+                              int(bool(causal)), _stream_ptr(stream))
+    if rc != OK:
+        raise NovaAttnError(rc, "nova_attn_fwd")
+
+
+def nova_attn_bwd_preprocess(O, dO, Delta, stream=None) -> None:
+    """Delta <- rowsum(dO * O)."""
+    _check_bf16("O", O)
+    _check_bf16("dO", dO, O.shape)
+    B, H, T, D = O.shape
+    _check_f32("Delta", Delta, (B, H, T))
+    rc = load().nova_attn_bwd_preprocess(_ptr(O), _ptr(dO), _ptr(Delta), B, H, T, D, _stream_ptr(stream))
+    if rc != OK:
+        raise NovaAttnError(rc, "nova_attn_bwd_preprocess")
+
+
+def nova_attn_bwd(Q, K, V, O, dO, LSE, Delta, dQ, dK, dV, scale: float, causal: bool = True, workspace=None,
+                  stream=None) -> None:
+    """dQ, dK, dV <- gradients of sum(O*dO); `workspace` is a CUDA byte/float tensor of at least
+    nova_attn_bwd_workspace_bytes(B,H,T,D) bytes (allocated here if omitted)."""
+    _check_bf16("Q", Q)
+    B, H, T, D = Q.shape
+    for n, t in (("K", K), ("V", V), ("O", O), ("dO", dO), ("dQ", dQ), ("dK", dK), ("dV", dV)):
+        _check_bf16(n, t, Q.shape)
+    _check_f32("LSE", LSE, (B, H, T))
+    _check_f32("Delta", Delta, (B, H, T))
+    if workspace is None:
+        workspace = torch.empty(nova_attn_bwd_workspace_bytes(B, H, T, D), dtype=torch.uint8, device=Q.device)
+    ws_bytes = workspace.numel() * workspace.element_size()
+    rc = load().nova_attn_bwd(_ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(dO), _ptr(LSE), _ptr(Delta), _ptr(dQ),
+                              _ptr(dK), _ptr(dV), B, H, T, D, float(scale), int(bool(causal)), _ptr(workspace),
+                              ws_bytes, _stream_ptr(stream))
+    if rc != OK:
+        raise NovaAttnError(rc, "nova_attn_bwd")
+
+
+def nova_attn_poll_device_status(stream=None) -> int:
+    """Synchronises the stream and returns the device status (0 = ok); raises on a recorded timeout."""
+    rc = load().nova_attn_poll_device_status(_stream_ptr(stream))
+    if rc != OK:
+        raise NovaAttnError(rc, "nova_attn_poll_device_status")
+    return rc
