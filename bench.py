@@ -1,0 +1,382 @@
+#!/usr/bin/env python
+"""Benchmark of the fused causal attention path (forward + backward preprocess + backward).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+One step = nova_attn_fwd + nova_attn_bwd_preprocess + nova_attn_bwd over one batch of the GPT-2-small
+training attention shape (B=8, H=12, T=1024, D=64, causal, bf16).  Prints ONE JSON line.
+
+  value      counted causal TFLOP/s (fwd 2*B*H*T^2*D, bwd 2.5x) of the whole job, inputs resident in
+             HBM, timed with CUDA events on the launching stream, max over ranks.
+  e2e        the same metric with the step's inputs copied from pinned host memory and its results
+             copied back inside the timed region.
+  roofline   tensor-core roofline of the dominant kernel (the fused backward), from a second pass
+             that brackets each kernel with events.
+  cpu_baseline  the fp64 oracle timed on the host cores on a bounded sample of the same workload.
+
+With N > 1 (launched by torchrun, one rank per GPU) every rank runs the same per-GPU batch on its own
+data: weak scaling, no data-path collective.  `--impl reference` times the CPU oracle instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+from paper_2608_00029_b200 import multi, workloads as W  # noqa: E402
+
+METRIC = "causal_attn_fwd_bwd_tflops"
+UNIT = "TFLOP/s"
+WORKLOAD = "gpt2_small"
+L2_BYTES = 126e6
+FALLBACK_PEAKS = {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            p = json.load(f)
+        return {k: float(p[k]) for k in FALLBACK_PEAKS}, "measured"
+    except Exception:
+        return dict(FALLBACK_PEAKS), "fallback"
+
+
+# ------------------------------------------------------------------------------------------ clocks
+class ClockSampler(threading.Thread):
+    """Samples SM clock, power and clock-event reasons through NVML (read-only) while the GPU works."""
+
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
+
+    def __init__(self, device_index: int, period_s: float = 0.01):
+        super().__init__(daemon=True)
+        self.period = period_s
+        self.samples = []  # (t, sm_mhz, reasons_mask, power_w)
+        self._halt = threading.Event()
+        self.ok = False
+        self.max_mhz = None
+        try:
+            import pynvml
+            self.nv = pynvml
+            pynvml.nvmlInit()
+            uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+            if not uuid.startswith("GPU-"):
+                uuid = "GPU-" + uuid
+            try:
+                self.h = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode())
+            except Exception:
+                self.h = pynvml.nvmlDeviceGetHandleByIndex(device_index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        while not self._halt.is_set():
+            try:
+                mhz = int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+                except Exception:
+                    mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                try:
+                    pw = nv.nvmlDeviceGetPowerUsage(self.h) / 1000.0
+                except Exception:
+                    pw = None
+                self.samples.append((time.perf_counter(), mhz, mask, pw))
+            except Exception:
+                pass
+            self._halt.wait(self.period)
+
+    def stop(self):
+        self._halt.set()
+
+    def summary(self, t0: float, t1: float) -> dict:
+        if not self.ok or not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0, "note": "NVML unavailable"}
+        inside = [s for s in self.samples if t0 <= s[0] <= t1]
+        note = "sampled during the timed region"
+        if len(inside) < 3:
+            busy = sorted(self.samples, key=lambda s: -(s[3] or 0))[: max(3, len(self.samples) // 4)]
+            inside = busy
+            note = "timed region shorter than the sampling period: highest-power samples of the whole run"
+        clocks = sorted(s[1] for s in inside)
+        mask = 0
+        for s in inside:
+            mask |= s[2]
+        reasons = [name for bit, name in self.REASONS.items() if mask & bit]
+        powers = [s[3] for s in inside if s[3] is not None]
+        return {"sm_mhz": clocks[len(clocks) // 2], "sm_max_mhz": self.max_mhz, "reasons": reasons,
+                "samples": len(inside), "power_w_max": max(powers) if powers else None, "note": note}
+
+
+# ------------------------------------------------------------------------------------------ oracle leg
+def time_oracle(cfg, Q, K, V, dO, budget_s: float = 12.0, max_batches: int | None = None):
+    """Times the fp64 CPU oracle (forward + backward) batch by batch until about `budget_s` seconds of
+    work are done.  Returns (TFLOP/s, threads, description of the sample)."""
+    import oracle
+    threads = oracle.num_threads()
+    per_batch_flops = (cfg.fwd_flops + cfg.bwd_flops) / cfg.B
+    done, spent = 0, 0.0
+    nb = cfg.B if max_batches is None else min(cfg.B, max_batches)
+    for b in range(nb):
+        q, k, v, do = (W.widen(x[b:b + 1]) for x in (Q, K, V, dO))
+        t0 = time.perf_counter()
+        oracle.attn_fwd(q, k, v, cfg.scale, cfg.causal)
+        oracle.attn_bwd(q, k, v, do, cfg.scale, cfg.causal)
+        spent += time.perf_counter() - t0
+        done += 1
+        if spent >= budget_s:
+            break
+    tflops = done * per_batch_flops / spent / 1e12
+    sample = f"{done} of {cfg.B} sequences ({done * cfg.H} heads) of {cfg.name}, fwd+bwd once, {spent:.2f} s"
+    return tflops, threads, sample, spent / done
+
+
+def run_reference(args):
+    """The reference arm of this build is the fp64 CPU oracle as it stands.  Each step runs it forward +
+    backward on a bounded sample of the workload: one whole sequence (all heads of one batch entry)
+    when K + W such steps fit in about four minutes, otherwise a single head."""
+    rank, _, world = multi.env_rank_world()
+    if rank != 0:
+        return 0
+    import oracle
+    oracle.build()
+    cfg = W.CONFIGS[WORKLOAD]
+    Q, K, V, dO = W.make_inputs(cfg)
+    threads = oracle.num_threads()
+
+    def run_sample(b, heads):
+        q, k, v, do = (W.widen(x[b:b + 1, :heads]) for x in (Q, K, V, dO))
+        oracle.attn_fwd(q, k, v, cfg.scale, cfg.causal)
+        oracle.attn_bwd(q, k, v, do, cfg.scale, cfg.causal)
+
+    t0 = time.perf_counter()
+    run_sample(0, cfg.H)  # calibration, untimed
+    t_seq = time.perf_counter() - t0
+    heads = cfg.H if t_seq * (args.steps + args.warmup) <= 240.0 else 1
+    for i in range(args.warmup):
+        run_sample(i % cfg.B, heads)
+    t0 = time.perf_counter()
+    for i in range(args.steps):
+        run_sample(i % cfg.B, heads)
+    dt = (time.perf_counter() - t0) / max(args.steps, 1)
+    flops = (cfg.fwd_flops + cfg.bwd_flops) / (cfg.B * cfg.H) * heads
+    value = flops / dt / 1e12
+    sample = f"{heads} of {cfg.B * cfg.H} heads of {cfg.name} per step, fwd+bwd"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": cfg.name, "B": cfg.B, "H": cfg.H, "T": cfg.T, "D": cfg.D, "causal": True,
+                   "note": "fp64 CPU oracle on the host cores; each step is a bounded sample of the workload"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": min(threads, heads), "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+    return 0
+
+
+# ------------------------------------------------------------------------------------------ our arm
+class BufferSet:
+    def __init__(self, cfg, dev, inputs):
+        from paper_2608_00029_b200 import nova_attn
+        self.q, self.k, self.v, self.do = (x.to(dev) for x in inputs)
+        shape = (cfg.B, cfg.H, cfg.T, cfg.D)
+        self.o, self.dq, self.dk, self.dv = (torch.empty(shape, dtype=torch.bfloat16, device=dev) for _ in range(4))
+        self.lse = torch.empty((cfg.B, cfg.H, cfg.T), dtype=torch.float32, device=dev)
+        self.delta = torch.empty_like(self.lse)
+        self.ws = torch.empty(nova_attn.nova_attn_bwd_workspace_bytes(*shape), dtype=torch.uint8, device=dev)
+
+    def bytes(self):
+        t = (self.q, self.k, self.v, self.do, self.o, self.dq, self.dk, self.dv, self.lse, self.delta, self.ws)
+        return sum(x.numel() * x.element_size() for x in t)
+
+
+def step(na, cfg, s):
+    na.nova_attn_fwd(s.q, s.k, s.v, s.o, s.lse, cfg.scale, cfg.causal)
+    na.nova_attn_bwd_preprocess(s.o, s.do, s.delta)
+    na.nova_attn_bwd(s.q, s.k, s.v, s.o, s.do, s.lse, s.delta, s.dq, s.dk, s.dv, cfg.scale, cfg.causal, s.ws)
+
+
+def run_ours(args):
+    from paper_2608_00029_b200 import nova_attn as na
+    na.load()  # fails loudly if the CUDA library has not been built
+    rank, local_rank, world = multi.env_rank_world()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the attention path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        multi.init_process_group("nccl")
+    peaks, peak_src = load_peaks()
+
+    base = W.CONFIGS[WORKLOAD]
+    plan = multi.weak_scaling_plan(base.B, world, rank)
+    cfg = base.replace(B=plan["local_batch"])
+    # Rotate over enough independent buffer sets that the data touched between two uses of the same
+    # set exceeds L2, so no step finds its inputs cached from the previous use.
+    probe = BufferSet(cfg, dev, W.make_inputs(cfg, seed=base.seed + 1000 * rank))
+    n_sets = max(2, int(L2_BYTES * 2 // probe.bytes()) + 2)
+    sets = [probe] + [BufferSet(cfg, dev, W.make_inputs(cfg, seed=base.seed + 1000 * rank + i)) for i in range(1, n_sets)]
+    stream = torch.cuda.current_stream()
+    flops_step = cfg.fwd_flops + cfg.bwd_flops
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+
+    # ---- device-resident timing
+    for i in range(max(args.warmup, 3)):
+        step(na, cfg, sets[i % n_sets])
+    torch.cuda.synchronize()
+    multi.barrier()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    t_region0 = time.perf_counter()
+    ev0.record(stream)
+    for i in range(args.steps):
+        step(na, cfg, sets[i % n_sets])
+    ev1.record(stream)
+    torch.cuda.synchronize()
+    t_region1 = time.perf_counter()
+    multi.barrier()
+    ms_total = multi.max_over_ranks(ev0.elapsed_time(ev1), dev)
+    na.nova_attn_poll_device_status()
+    ms_per_step = ms_total / args.steps
+    value = flops_step * world / (ms_per_step * 1e-3) / 1e12
+
+    # ---- per-kernel attribution (separate pass, same rotation): events around each launch
+    names = ["fwd", "bwd_preprocess", "bwd_zero", "bwd_main", "bwd_convert"]
+    k_steps = min(args.steps, 200)
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(len(names) + 1)] for _ in range(k_steps)]
+    for i in range(k_steps):
+        s = sets[i % n_sets]
+        e = evs[i]
+        e[0].record(stream)
+        na.nova_attn_fwd(s.q, s.k, s.v, s.o, s.lse, cfg.scale, cfg.causal)
+        e[1].record(stream)
+        na.nova_attn_bwd_preprocess(s.o, s.do, s.delta)
+        e[2].record(stream)
+        for n, bit in enumerate((na.BWD_STEP_ZERO, na.BWD_STEP_MAIN, na.BWD_STEP_CONVERT)):
+            na.nova_attn_bwd(s.q, s.k, s.v, s.o, s.do, s.lse, s.delta, s.dq, s.dk, s.dv, cfg.scale, cfg.causal, s.ws,
+                             steps=bit)
+            e[3 + n].record(stream)
+    torch.cuda.synchronize()
+    kernel_ms = {n: sum(e[i].elapsed_time(e[i + 1]) for e in evs) / k_steps for i, n in enumerate(names)}
+    bwd_ms = kernel_ms["bwd_main"]
+    achieved = cfg.bwd_flops / (bwd_ms * 1e-3) / 1e12
+    # a kernel timed inside a long back-to-back run is compared with the sustained GEMM figure
+    peak = peaks["bf16_tflops_sustained"]
+    roofline = {
+        "bound": "tensor", "kernel": "attn_bwd_kernel", "achieved": achieved, "peak": peak, "unit": UNIT,
+        "frac": achieved / peak, "traffic": None, "peak_source": f"{peak_src} bf16_tflops_sustained",
+        "frac_of_burst_peak": achieved / peaks["bf16_tflops"], "ms_per_launch": bwd_ms,
+        "kernel_ms": kernel_ms,
+        "fwd_tflops": cfg.fwd_flops / (kernel_ms["fwd"] * 1e-3) / 1e12,
+        "fwd_frac_of_burst_peak": cfg.fwd_flops / (kernel_ms["fwd"] * 1e-3) / 1e12 / peaks["bf16_tflops"],
+        "preprocess_gbs": (4.0 * cfg.B * cfg.H * cfg.T * cfg.D + 4.0 * cfg.B * cfg.H * cfg.T)
+        / (kernel_ms["bwd_preprocess"] * 1e-3) / 1e9,
+    }
+    traffic_path = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(traffic_path):
+        try:
+            with open(traffic_path) as f:
+                roofline["traffic"] = json.load(f).get("attn_bwd_kernel_bytes_per_launch")
+        except Exception:
+            pass
+
+    # ---- end to end: pinned host inputs in, results out, every step
+    host_in = [tuple(x.pin_memory() for x in W.make_inputs(cfg, seed=base.seed + 1000 * rank + 7)) for _ in range(2)]
+    host_out = [tuple(torch.empty((cfg.B, cfg.H, cfg.T, cfg.D), dtype=torch.bfloat16).pin_memory() for _ in range(4))
+                for _ in range(2)]
+    h2d = sum(x.numel() * x.element_size() for x in host_in[0])
+    d2h = sum(x.numel() * x.element_size() for x in host_out[0])
+
+    def e2e_step(i):
+        s = sets[i % n_sets]
+        hi, ho = host_in[i % 2], host_out[i % 2]
+        for dst, src in zip((s.q, s.k, s.v, s.do), hi):
+            dst.copy_(src, non_blocking=True)
+        step(na, cfg, s)
+        for dst, src in zip(ho, (s.o, s.dq, s.dk, s.dv)):
+            dst.copy_(src, non_blocking=True)
+
+    e2e_steps = max(3, min(args.steps, 50))
+    for i in range(3):
+        e2e_step(i)
+    torch.cuda.synchronize()
+    multi.barrier()
+    ev0.record(stream)
+    for i in range(e2e_steps):
+        e2e_step(i)
+    ev1.record(stream)
+    torch.cuda.synchronize()
+    multi.barrier()
+    e2e_ms = multi.max_over_ranks(ev0.elapsed_time(ev1), dev) / e2e_steps
+    e2e_value = flops_step * world / (e2e_ms * 1e-3) / 1e12
+    na.nova_attn_poll_device_status()
+
+    sampler.stop()
+    sampler.join(timeout=2)
+    clocks = sampler.summary(t_region0, t_region1)
+
+    cpu_baseline = None
+    if rank == 0 and world == 1:
+        import oracle
+        oracle.build()
+        inputs = W.make_inputs(base)
+        v, threads, sample, _ = time_oracle(base, *inputs, budget_s=12.0)
+        cpu_baseline = {"value": v, "unit": UNIT, "cores": min(threads, base.H), "kind": "oracle", "sample": sample}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": base.name, "B_per_gpu": cfg.B, "global_batch": plan["global_batch"], "H": cfg.H,
+                       "T": cfg.T, "D": cfg.D, "causal": True, "parallelism": f"dp{world} (batch split, no collective)",
+                       "l2": f"rotating {n_sets} buffer sets of {probe.bytes() / 1e6:.0f} MB "
+                             f"({n_sets * probe.bytes() / 1e6:.0f} MB > 126 MB L2)",
+                       "flops_per_step": flops_step, "frac_of_burst_peak": value / world / peaks["bf16_tflops"]},
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "ms_per_step": e2e_ms, "steps": e2e_steps},
+            "gpu_launches": 4 * args.steps,
+            "clocks": clocks,
+            "roofline": roofline,
+            "cpu_baseline": cpu_baseline,
+        }
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        multi.barrier()
+        torch.distributed.destroy_process_group()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=500)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

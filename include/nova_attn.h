@@ -71,6 +71,23 @@ int nova_attn_bwd_preprocess(const void* O, const void* dO, float* Delta,
                              int B, int H, int T, int D, void* stream);
 
 /*
+ * Exact variant of the preprocess: Delta_i = sum_j P_ij * (dO_i . V_j) over the kept keys, with P
+ * rebuilt from LSE inside the kernel (paper Section 4.2, "The Backward Pass": the probability matrix
+ * is recomputed from the cached log-sum-exp, never stored).  Mathematically equal to rowsum(dO * O),
+ * but independent of the bf16 rounding of the stored O: rowsum(dO * O) carries an error of about
+ * 2^-9 * sum_d |dO_d O_d|, which reaches dQ and dK multiplied by scale * |sum_j P_ij K_j| and
+ * dominates their error when softmax rows are sharply peaked (|O| ~ |V|).  Costs two extra
+ * contractions and one exp2 per score, i.e. roughly one forward pass.  Use it in place of
+ * nova_attn_bwd_preprocess when that accuracy matters; nova_attn_bwd accepts either Delta.
+ *   Q, K, V, dO : in,  bf16 [B,H,T,D]
+ *   LSE         : in,  fp32 [B,H,T] from nova_attn_fwd
+ *   Delta       : out, fp32 [B,H,T]
+ */
+int nova_attn_bwd_preprocess_exact(const void* Q, const void* K, const void* V, const void* dO,
+                                   const float* LSE, float* Delta, int B, int H, int T, int D,
+                                   float scale, int causal, void* stream);
+
+/*
  * Bytes of scratch nova_attn_bwd needs: an fp32 accumulator for dQ, [B,H,T,D].
  * Returns 0 if the shape is invalid.
  */
@@ -93,6 +110,23 @@ int nova_attn_bwd(const void* Q, const void* K, const void* V, const void* O, co
                   const float* LSE, const float* Delta, void* dQ, void* dK, void* dV,
                   int B, int H, int T, int D, float scale, int causal,
                   void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * The three steps nova_attn_bwd enqueues, selectable one by one so that each can be timed alone
+ * (a measurement aid: the paper has no counterpart).  `steps` is a bit mask:
+ *   NOVA_ATTN_BWD_STEP_ZERO     clear the fp32 dQ accumulator in `workspace`
+ *   NOVA_ATTN_BWD_STEP_MAIN     the fused backward kernel: writes dK, dV, accumulates unscaled dQ
+ *   NOVA_ATTN_BWD_STEP_CONVERT  dQ = bf16(scale * accumulator)
+ * All three, in this order, are what nova_attn_bwd does; any other combination leaves sequencing to
+ * the caller.  Arguments, validation and errors are those of nova_attn_bwd.
+ */
+#define NOVA_ATTN_BWD_STEP_ZERO 1
+#define NOVA_ATTN_BWD_STEP_MAIN 2
+#define NOVA_ATTN_BWD_STEP_CONVERT 4
+int nova_attn_bwd_steps(const void* Q, const void* K, const void* V, const void* O, const void* dO,
+                        const float* LSE, const float* Delta, void* dQ, void* dK, void* dV,
+                        int B, int H, int T, int D, float scale, int causal,
+                        void* workspace, size_t workspace_bytes, void* stream, int steps);
 
 /* Static, never-freed description of a status code. */
 const char* nova_attn_status_string(int status);

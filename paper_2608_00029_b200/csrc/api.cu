@@ -69,6 +69,7 @@ int device_state(DeviceState** out) {
         }
         e = configure_attn_fwd();
         if (e == cudaSuccess) e = configure_attn_bwd();
+        if (e == cudaSuccess) e = configure_attn_delta();
         if (e == cudaSuccess) e = cudaGetSymbolAddress(reinterpret_cast<void**>(&st.dev_status), g_dev_status);
         if (e != cudaSuccess) { st.status = fail_cuda(e); return st.status; }
     }
@@ -171,14 +172,35 @@ int nova_attn_bwd_preprocess(const void* O, const void* dO, float* Delta, int B,
     return e == cudaSuccess ? NOVA_ATTN_OK : fail_cuda(e);
 }
 
+int nova_attn_bwd_preprocess_exact(const void* Q, const void* K, const void* V, const void* dO, const float* LSE,
+                                   float* Delta, int B, int H, int T, int D, float scale, int causal, void* stream) {
+    if (!Q || !K || !V || !dO || !LSE || !Delta) return NOVA_ATTN_ERR_NULL;
+    if (int rc = check_shape(B, H, T, D)) return rc;
+    if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(dO) || !aligned16(LSE) || !aligned16(Delta))
+        return NOVA_ATTN_ERR_ALIGNMENT;
+    if (!std::isfinite(scale) || !(scale > 0.f)) return NOVA_ATTN_ERR_SCALE;
+    DeviceState* st = nullptr;
+    if (int rc = device_state(&st)) return rc;
+    const long long BH = static_cast<long long>(B) * H;
+    CUtensorMap tmQ, tmK, tmV, tmdO;
+    if (int rc = get_tensor_map(Q, D, T, BH, &tmQ)) return rc;
+    if (int rc = get_tensor_map(K, D, T, BH, &tmK)) return rc;
+    if (int rc = get_tensor_map(V, D, T, BH, &tmV)) return rc;
+    if (int rc = get_tensor_map(dO, D, T, BH, &tmdO)) return rc;
+    const AttnShape s{B, H, T, D, causal != 0, scale};
+    const cudaError_t e =
+        launch_attn_delta(tmQ, tmK, tmV, tmdO, LSE, Delta, s, st->dev_status, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? NOVA_ATTN_OK : fail_cuda(e);
+}
+
 size_t nova_attn_bwd_workspace_bytes(int B, int H, int T, int D) {
     if (check_shape(B, H, T, D) != NOVA_ATTN_OK) return 0;
     return static_cast<size_t>(B) * H * T * D * sizeof(float);
 }
 
-int nova_attn_bwd(const void* Q, const void* K, const void* V, const void* O, const void* dO, const float* LSE,
-                  const float* Delta, void* dQ, void* dK, void* dV, int B, int H, int T, int D, float scale,
-                  int causal, void* workspace, size_t workspace_bytes, void* stream) {
+int nova_attn_bwd_steps(const void* Q, const void* K, const void* V, const void* O, const void* dO, const float* LSE,
+                        const float* Delta, void* dQ, void* dK, void* dV, int B, int H, int T, int D, float scale,
+                        int causal, void* workspace, size_t workspace_bytes, void* stream, int steps) {
     (void)O;  // Delta already carries rowsum(dO * O)
     if (!Q || !K || !V || !dO || !LSE || !Delta || !dQ || !dK || !dV) return NOVA_ATTN_ERR_NULL;
     if (int rc = check_shape(B, H, T, D)) return rc;
@@ -192,22 +214,38 @@ int nova_attn_bwd(const void* Q, const void* K, const void* V, const void* O, co
     DeviceState* st = nullptr;
     if (int rc = device_state(&st)) return rc;
     const long long BH = static_cast<long long>(B) * H;
-    CUtensorMap tmQ, tmK, tmV, tmdO;
-    if (int rc = get_tensor_map(Q, D, T, BH, &tmQ)) return rc;
-    if (int rc = get_tensor_map(K, D, T, BH, &tmK)) return rc;
-    if (int rc = get_tensor_map(V, D, T, BH, &tmV)) return rc;
-    if (int rc = get_tensor_map(dO, D, T, BH, &tmdO)) return rc;
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     float* acc = static_cast<float*>(workspace);
-    cudaError_t e = cudaMemsetAsync(acc, 0, need, cs);
-    if (e != cudaSuccess) return fail_cuda(e);
-    const AttnShape s{B, H, T, D, causal != 0, scale};
-    e = launch_attn_bwd(tmQ, tmK, tmV, tmdO, LSE, Delta, acc, static_cast<__nv_bfloat16*>(dK),
-                        static_cast<__nv_bfloat16*>(dV), s, st->dev_status, cs);
-    if (e != cudaSuccess) return fail_cuda(e);
-    e = launch_dq_convert(acc, static_cast<__nv_bfloat16*>(dQ), static_cast<long long>(need / sizeof(float)), scale,
-                          st->num_sms, cs);
-    return e == cudaSuccess ? NOVA_ATTN_OK : fail_cuda(e);
+    cudaError_t e = cudaSuccess;
+    if (steps & NOVA_ATTN_BWD_STEP_ZERO) {
+        e = cudaMemsetAsync(acc, 0, need, cs);
+        if (e != cudaSuccess) return fail_cuda(e);
+    }
+    if (steps & NOVA_ATTN_BWD_STEP_MAIN) {
+        CUtensorMap tmQ, tmK, tmV, tmdO;
+        if (int rc = get_tensor_map(Q, D, T, BH, &tmQ)) return rc;
+        if (int rc = get_tensor_map(K, D, T, BH, &tmK)) return rc;
+        if (int rc = get_tensor_map(V, D, T, BH, &tmV)) return rc;
+        if (int rc = get_tensor_map(dO, D, T, BH, &tmdO)) return rc;
+        const AttnShape s{B, H, T, D, causal != 0, scale};
+        e = launch_attn_bwd(tmQ, tmK, tmV, tmdO, LSE, Delta, acc, static_cast<__nv_bfloat16*>(dK),
+                            static_cast<__nv_bfloat16*>(dV), s, st->dev_status, cs);
+        if (e != cudaSuccess) return fail_cuda(e);
+    }
+    if (steps & NOVA_ATTN_BWD_STEP_CONVERT) {
+        e = launch_dq_convert(acc, static_cast<__nv_bfloat16*>(dQ), static_cast<long long>(need / sizeof(float)),
+                              scale, st->num_sms, cs);
+        if (e != cudaSuccess) return fail_cuda(e);
+    }
+    return NOVA_ATTN_OK;
+}
+
+int nova_attn_bwd(const void* Q, const void* K, const void* V, const void* O, const void* dO, const float* LSE,
+                  const float* Delta, void* dQ, void* dK, void* dV, int B, int H, int T, int D, float scale,
+                  int causal, void* workspace, size_t workspace_bytes, void* stream) {
+    return nova_attn_bwd_steps(Q, K, V, O, dO, LSE, Delta, dQ, dK, dV, B, H, T, D, scale, causal, workspace,
+                               workspace_bytes, stream,
+                               NOVA_ATTN_BWD_STEP_ZERO | NOVA_ATTN_BWD_STEP_MAIN | NOVA_ATTN_BWD_STEP_CONVERT);
 }
 
 const char* nova_attn_status_string(int status) {

@@ -28,6 +28,12 @@ cudaError_t configure_attn_fwd();
 cudaError_t launch_attn_bwd_preprocess(const __nv_bfloat16* O, const __nv_bfloat16* dO, float* Delta,
                                        long long rows, int D, int num_sms, cudaStream_t stream);
 
+// Exact Delta_i = sum_j P_ij (dO_i . V_j) with P rebuilt from LSE (two contractions + exp2 per tile).
+cudaError_t launch_attn_delta(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV,
+                              const CUtensorMap& tmdO, const float* LSE, float* Delta, const AttnShape& s,
+                              int* dev_status, cudaStream_t stream);
+cudaError_t configure_attn_delta();
+
 // Backward main kernel: accumulates unscaled dQ into `dq_acc` (fp32 [B,H,T,D], zeroed beforehand),
 // writes dK and dV.
 cudaError_t launch_attn_bwd(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV,

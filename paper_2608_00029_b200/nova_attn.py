@@ -43,10 +43,14 @@ def load():
     lib.nova_attn_fwd.restype = i
     lib.nova_attn_bwd_preprocess.argtypes = [vp, vp, fp, i, i, i, i, vp]
     lib.nova_attn_bwd_preprocess.restype = i
+    lib.nova_attn_bwd_preprocess_exact.argtypes = [vp, vp, vp, vp, fp, fp, i, i, i, i, f, i, vp]
+    lib.nova_attn_bwd_preprocess_exact.restype = i
     lib.nova_attn_bwd_workspace_bytes.argtypes = [i, i, i, i]
     lib.nova_attn_bwd_workspace_bytes.restype = sz
     lib.nova_attn_bwd.argtypes = [vp] * 5 + [fp, fp, vp, vp, vp, i, i, i, i, f, i, vp, sz, vp]
     lib.nova_attn_bwd.restype = i
+    lib.nova_attn_bwd_steps.argtypes = [vp] * 5 + [fp, fp, vp, vp, vp, i, i, i, i, f, i, vp, sz, vp, i]
+    lib.nova_attn_bwd_steps.restype = i
     lib.nova_attn_status_string.argtypes = [i]
     lib.nova_attn_status_string.restype = ctypes.c_char_p
     lib.nova_attn_last_cuda_error.argtypes = []
@@ -116,10 +120,29 @@ def nova_attn_bwd_preprocess(O, dO, Delta, stream=None) -> None:
         raise NovaAttnError(rc, "nova_attn_bwd_preprocess")
 
 
+def nova_attn_bwd_preprocess_exact(Q, K, V, dO, LSE, Delta, scale: float, causal: bool = True, stream=None) -> None:
+    """Delta <- sum_j P_ij (dO_i . V_j) with P rebuilt from LSE: independent of the rounding of O."""
+    _check_bf16("Q", Q)
+    B, H, T, D = Q.shape
+    for n, t in (("K", K), ("V", V), ("dO", dO)):
+        _check_bf16(n, t, Q.shape)
+    _check_f32("LSE", LSE, (B, H, T))
+    _check_f32("Delta", Delta, (B, H, T))
+    rc = load().nova_attn_bwd_preprocess_exact(_ptr(Q), _ptr(K), _ptr(V), _ptr(dO), _ptr(LSE), _ptr(Delta), B, H, T,
+                                               D, float(scale), int(bool(causal)), _stream_ptr(stream))
+    if rc != OK:
+        raise NovaAttnError(rc, "nova_attn_bwd_preprocess_exact")
+
+
+BWD_STEP_ZERO, BWD_STEP_MAIN, BWD_STEP_CONVERT = 1, 2, 4
+BWD_STEP_ALL = 7
+
+
 def nova_attn_bwd(Q, K, V, O, dO, LSE, Delta, dQ, dK, dV, scale: float, causal: bool = True, workspace=None,
-                  stream=None) -> None:
+                  stream=None, steps: int = BWD_STEP_ALL) -> None:
     """dQ, dK, dV <- gradients of sum(O*dO); `workspace` is a CUDA byte/float tensor of at least
-    nova_attn_bwd_workspace_bytes(B,H,T,D) bytes (allocated here if omitted)."""
+    nova_attn_bwd_workspace_bytes(B,H,T,D) bytes (allocated here if omitted).  `steps` other than
+    BWD_STEP_ALL goes through nova_attn_bwd_steps (a timing aid)."""
     _check_bf16("Q", Q)
     B, H, T, D = Q.shape
     for n, t in (("K", K), ("V", V), ("O", O), ("dO", dO), ("dQ", dQ), ("dK", dK), ("dV", dV)):
@@ -129,9 +152,12 @@ def nova_attn_bwd(Q, K, V, O, dO, LSE, Delta, dQ, dK, dV, scale: float, causal: 
     if workspace is None:
         workspace = torch.empty(nova_attn_bwd_workspace_bytes(B, H, T, D), dtype=torch.uint8, device=Q.device)
     ws_bytes = workspace.numel() * workspace.element_size()
-    rc = load().nova_attn_bwd(_ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(dO), _ptr(LSE), _ptr(Delta), _ptr(dQ),
-                              _ptr(dK), _ptr(dV), B, H, T, D, float(scale), int(bool(causal)), _ptr(workspace),
-                              ws_bytes, _stream_ptr(stream))
+    args = (_ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(dO), _ptr(LSE), _ptr(Delta), _ptr(dQ), _ptr(dK), _ptr(dV),
+            B, H, T, D, float(scale), int(bool(causal)), _ptr(workspace), ws_bytes, _stream_ptr(stream))
+    if steps == BWD_STEP_ALL:
+        rc = load().nova_attn_bwd(*args)
+    else:
+        rc = load().nova_attn_bwd_steps(*args, int(steps))
     if rc != OK:
         raise NovaAttnError(rc, "nova_attn_bwd")
 

@@ -17,9 +17,10 @@ def _guarded(shape, dtype, dev, fill):
     return buf, buf[GUARD:GUARD + n].view(shape)
 
 
-def run_gpu(Q, K, V, dO, scale, causal=True, O_in=None, LSE_in=None, check_guards=True):
+def run_gpu(Q, K, V, dO, scale, causal=True, O_in=None, LSE_in=None, check_guards=True, exact_delta=False):
     """Forward + preprocess + backward on cuda:0.  Returns CPU tensors.  If O_in/LSE_in are given the
-    backward consumes them instead of the forward's own results."""
+    backward consumes them instead of the forward's own results.  `exact_delta` selects
+    nova_attn_bwd_preprocess_exact (Delta from P and dO V^T) instead of rowsum(dO * O)."""
     dev = torch.device("cuda:0")
     q, k, v, do = (x.to(dev).contiguous() for x in (Q, K, V, dO))
     B, H, T, D = q.shape
@@ -32,7 +33,10 @@ def run_gpu(Q, K, V, dO, scale, causal=True, O_in=None, LSE_in=None, check_guard
     nova_attn.nova_attn_fwd(q, k, v, views["O"], views["LSE"], scale, causal)
     o_b = views["O"] if O_in is None else O_in.to(dev)
     lse_b = views["LSE"] if LSE_in is None else LSE_in.to(dev)
-    nova_attn.nova_attn_bwd_preprocess(o_b, do, views["Delta"])
+    if exact_delta:
+        nova_attn.nova_attn_bwd_preprocess_exact(q, k, v, do, lse_b, views["Delta"], scale, causal)
+    else:
+        nova_attn.nova_attn_bwd_preprocess(o_b, do, views["Delta"])
     nova_attn.nova_attn_bwd(q, k, v, o_b, do, lse_b, views["Delta"], views["dQ"], views["dK"], views["dV"],
                             scale, causal)
     nova_attn.nova_attn_poll_device_status()
@@ -51,7 +55,7 @@ def run_oracle(Q, K, V, dO, scale, causal=True, heads=None):
     Qd, Kd, Vd, dOd = (W.widen(x) for x in (Q, K, V, dO))
     O, LSE = oracle.attn_fwd(Qd, Kd, Vd, scale, causal)
     dQ, dK, dV, Delta = oracle.attn_bwd(Qd, Kd, Vd, dOd, scale, causal)
-    return {"O": O, "LSE": LSE, "dQ": dQ, "dK": dK, "dV": dV, "Delta": Delta}
+    return {"O": O, "LSE": LSE, "dQ": dQ, "dK": dK, "dV": dV, "Delta": Delta, "dO_in": dOd}
 
 
 def select_heads(got, heads):
@@ -60,14 +64,24 @@ def select_heads(got, heads):
     return {n: W.widen(torch.stack([t[b, h] for b, h in heads]).unsqueeze(1)) for n, t in got.items()}
 
 
-def compare(got, ref, label="", rms=True):
-    """Element-wise bounds: O, LSE, Delta 1e-2 + 1e-2|ref|; dQ, dK, dV 2e-2 + 2e-2|ref|; plus relative
-    RMS bounds.  Returns the max abs errors."""
+def compare(got, ref, label="", rms=True, dO=None, bwd_factor=1.0):
+    """Element-wise bounds: O, LSE 1e-2 + 1e-2|ref|; dQ, dK, dV 2e-2 + 2e-2|ref|; plus relative RMS
+    bounds.  Delta is a D-term dot product of dO with the bf16 O the forward wrote, so its bound is the
+    forward bound pushed through that sum: 1e-2 + 1e-2 * sum_d |dO_d| |O_d|  (needs dO [.., T, D] as
+    float64; without it Delta is only checked by relative RMS).  Returns the max abs errors."""
     out = {}
-    for name in ("O", "LSE", "Delta"):
+    for name in ("O", "LSE"):
         out[name] = tol.assert_close(got[name], ref[name], tol.FWD_ATOL, tol.FWD_RTOL, f"{label}{name}",
                                      tol.FWD_REL_RMS if rms else None)
+    derr = np.abs(np.asarray(got["Delta"], dtype=np.float64) - ref["Delta"])
+    assert np.isfinite(got["Delta"]).all()
+    if dO is not None:
+        bound = tol.FWD_ATOL + tol.FWD_RTOL * (np.abs(dO) * np.abs(ref["O"])).sum(-1)
+        assert (derr <= bound).all(), f"{label}Delta: max|err|={derr.max():.3e} exceeds the propagated forward bound"
+    assert tol.rel_rms(got["Delta"], ref["Delta"]) <= tol.FWD_REL_RMS, f"{label}Delta relative RMS"
+    out["Delta"] = float(derr.max())
     for name in ("dQ", "dK", "dV"):
-        out[name] = tol.assert_close(got[name], ref[name], tol.BWD_ATOL, tol.BWD_RTOL, f"{label}{name}",
+        out[name] = tol.assert_close(got[name], ref[name], bwd_factor * tol.BWD_ATOL, bwd_factor * tol.BWD_RTOL,
+                                     f"{label}{name}",
                                      tol.BWD_REL_RMS if rms else None)
     return out

@@ -1,0 +1,83 @@
+"""The C-ABI library loads, exports every symbol the header declares, and validates arguments on the
+host before touching the GPU (no compute call is made here)."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+HEADER = os.path.join(ROOT, "include", "nova_attn.h")
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2608_00029_b200 import build, nova_attn
+    build.build()
+    return nova_attn.load()
+
+
+def _declared_symbols():
+    text = open(HEADER).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(nova_attn_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_header_symbols_are_exported(lib):
+    names = _declared_symbols()
+    assert {"nova_attn_fwd", "nova_attn_bwd_preprocess", "nova_attn_bwd", "nova_attn_bwd_workspace_bytes",
+            "nova_attn_status_string", "nova_attn_poll_device_status"} <= set(names)
+    for n in names:
+        assert hasattr(lib, n), f"{n} declared in nova_attn.h but not exported"
+
+
+def test_status_strings(lib):
+    from paper_2608_00029_b200 import nova_attn as na
+    assert na.nova_attn_status_string(0) == "ok"
+    seen = {na.nova_attn_status_string(c) for c in range(-8, 1)}
+    assert len(seen) == 9 and "unknown status" not in seen
+    assert na.nova_attn_status_string(-99) == "unknown status"
+
+
+def test_workspace_query(lib):
+    from paper_2608_00029_b200 import nova_attn as na
+    assert na.nova_attn_bwd_workspace_bytes(8, 12, 1024, 64) == 8 * 12 * 1024 * 64 * 4
+    assert na.nova_attn_bwd_workspace_bytes(2, 12, 8192, 128) == 2 * 12 * 8192 * 128 * 4
+    assert na.nova_attn_bwd_workspace_bytes(1, 1, 1, 96) == 0      # unsupported head dim
+    assert na.nova_attn_bwd_workspace_bytes(0, 1, 1, 64) == 0
+
+
+def test_host_side_validation_rejects_before_launch(lib):
+    from paper_2608_00029_b200 import nova_attn as na
+    p = ctypes.c_void_p(0x1000)       # aligned, never dereferenced: every case fails validation first
+    odd = ctypes.c_void_p(0x1008)
+    f = lib.nova_attn_fwd
+    assert f(None, p, p, p, p, 1, 1, 1, 64, 1.0, 1, None) == na.ERR_NULL
+    assert f(p, p, p, p, p, 0, 1, 1, 64, 1.0, 1, None) == na.ERR_SHAPE
+    assert f(p, p, p, p, p, 1, 1, -5, 64, 1.0, 1, None) == na.ERR_SHAPE
+    assert f(p, p, p, p, p, 1, 1, 16, 96, 1.0, 1, None) == na.ERR_UNSUPPORTED
+    assert f(p, odd, p, p, p, 1, 1, 16, 64, 1.0, 1, None) == na.ERR_ALIGNMENT
+    assert f(p, p, p, p, p, 1, 1, 16, 64, 0.0, 1, None) == na.ERR_SCALE
+    assert f(p, p, p, p, p, 1, 1, 16, 64, float("nan"), 1, None) == na.ERR_SCALE
+    assert f(p, p, p, p, p, 1, 1, 16, 64, float("inf"), 1, None) == na.ERR_SCALE
+    g = lib.nova_attn_bwd_preprocess
+    assert g(p, None, p, 1, 1, 1, 64, None) == na.ERR_NULL
+    assert g(p, p, p, 1, 1, 1, 32, None) == na.ERR_UNSUPPORTED
+    b = lib.nova_attn_bwd
+    args = [p] * 10
+    assert b(*args, 1, 1, 16, 64, 1.0, 1, None, 0, None) == na.ERR_WORKSPACE
+    assert b(*args, 1, 1, 16, 64, 1.0, 1, p, 16, None) == na.ERR_WORKSPACE      # too small
+    assert b(*args, 1, 1, 16, 64, -1.0, 1, p, 1 << 20, None) == na.ERR_SCALE
+    args[3] = None                                                              # O may be NULL: it is ignored
+    assert b(*args, 1, 1, 16, 64, 1.0, 1, p, 16, None) == na.ERR_WORKSPACE
+    e = lib.nova_attn_bwd_preprocess_exact
+    assert e(p, p, p, p, None, p, 1, 1, 16, 64, 1.0, 1, None) == na.ERR_NULL
+    assert e(p, p, p, p, p, p, 1, 1, 16, 64, -2.0, 1, None) == na.ERR_SCALE
+
+
+def test_missing_library_fails_loudly(monkeypatch, tmp_path):
+    from paper_2608_00029_b200 import nova_attn as na
+    monkeypatch.setattr(na, "_lib", None)
+    monkeypatch.setattr(na, "LIB_PATH", str(tmp_path / "libnova_attn.so"))
+    with pytest.raises(ImportError):
+        na.load()
