@@ -128,6 +128,34 @@ int nova_attn_bwd_steps(const void* Q, const void* K, const void* V, const void*
                         int B, int H, int T, int D, float scale, int causal,
                         void* workspace, size_t workspace_bytes, void* stream, int steps);
 
+/*
+ * Backward pass for callers that cannot allocate device memory (the paper has no counterpart).
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits - inside another framework's fixed
+ * memory plan, in a plugin that only ever sees its input and output buffers, or in a loop that must
+ * not touch the allocator once it is running.  Such callers cannot provide the `workspace` of
+ * nova_attn_bwd.  This variant takes the same inputs and outputs and keeps the fp32 dQ accumulator in
+ * a fixed array inside the library instead.
+ *
+ *   - The array holds nova_attn_static_scratch_bytes() = 32 MiB, i.e. B*H*T*D <= 8 Mi elements (the
+ *     GPT-2-small training shape B=8, H=12, T=1024, D=64 fits).  Larger problems are rejected with
+ *     NOVA_ATTN_ERR_WORKSPACE before anything is launched; use nova_attn_bwd for those.
+ *   - The array is part of the library image: every GPU that loads the library holds the 32 MiB until
+ *     the process exits, whether or not this function is ever called.
+ *   - The call allocates nothing: no cudaMalloc, no cudaFree, no allocating library routine.
+ *   - The first call on a device looks up the array's device address (one runtime query, cached per
+ *     device).  Make that first call before starting any stream capture.
+ *   - All calls on a device share the one array.  Each call clears the part it uses before use, so
+ *     what an earlier call left behind is harmless, but two calls whose GPU work overlaps (different
+ *     streams, or different host threads) race on it and corrupt each other's dQ.  Serialise them.
+ *   - Arguments, validation, results and error codes are otherwise those of nova_attn_bwd.
+ */
+size_t nova_attn_static_scratch_bytes(void);
+int nova_attn_bwd_static_scratch(const void* Q, const void* K, const void* V, const void* O,
+                                 const void* dO, const float* LSE, const float* Delta,
+                                 void* dQ, void* dK, void* dV, int B, int H, int T, int D,
+                                 float scale, int causal, void* stream);
+
 /* Static, never-freed description of a status code. */
 const char* nova_attn_status_string(int status);
 

@@ -57,11 +57,10 @@ def load():
     lib.nova_attn_last_cuda_error.restype = i
     lib.nova_attn_poll_device_status.argtypes = [vp]
     lib.nova_attn_poll_device_status.restype = i
-    if hasattr(lib, "nova_attn_bwd_static_scratch"):
-        lib.nova_attn_bwd_static_scratch.argtypes = [vp] * 5 + [fp, fp, vp, vp, vp, i, i, i, i, f, i, vp]
-        lib.nova_attn_bwd_static_scratch.restype = i
-        lib.nova_attn_static_scratch_bytes.argtypes = []
-        lib.nova_attn_static_scratch_bytes.restype = sz
+    lib.nova_attn_bwd_static_scratch.argtypes = [vp] * 5 + [fp, fp, vp, vp, vp, i, i, i, i, f, i, vp]
+    lib.nova_attn_bwd_static_scratch.restype = i
+    lib.nova_attn_static_scratch_bytes.argtypes = []
+    lib.nova_attn_static_scratch_bytes.restype = sz
     _lib = lib
     return lib
 
@@ -160,6 +159,30 @@ def nova_attn_bwd(Q, K, V, O, dO, LSE, Delta, dQ, dK, dV, scale: float, causal: 
         rc = load().nova_attn_bwd_steps(*args, int(steps))
     if rc != OK:
         raise NovaAttnError(rc, "nova_attn_bwd")
+
+
+def nova_attn_static_scratch_bytes() -> int:
+    """Size of the library's built-in dQ accumulator (bytes)."""
+    return int(load().nova_attn_static_scratch_bytes())
+
+
+def nova_attn_bwd_static_scratch(Q, K, V, O, dO, LSE, Delta, dQ, dK, dV, scale: float, causal: bool = True,
+                                 stream=None) -> None:
+    """nova_attn_bwd for callers that cannot allocate: no workspace argument, nothing is allocated here
+    or in the library.  The dQ accumulator is a fixed 32 MiB array inside the library, shared by all
+    calls on the device, so B*H*T*D must not exceed 8 Mi elements and calls must not overlap on the
+    GPU.  Make the first call on a device before any stream capture."""
+    _check_bf16("Q", Q)
+    B, H, T, D = Q.shape
+    for n, t in (("K", K), ("V", V), ("O", O), ("dO", dO), ("dQ", dQ), ("dK", dK), ("dV", dV)):
+        _check_bf16(n, t, Q.shape)
+    _check_f32("LSE", LSE, (B, H, T))
+    _check_f32("Delta", Delta, (B, H, T))
+    rc = load().nova_attn_bwd_static_scratch(_ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(dO), _ptr(LSE), _ptr(Delta),
+                                             _ptr(dQ), _ptr(dK), _ptr(dV), B, H, T, D, float(scale),
+                                             int(bool(causal)), _stream_ptr(stream))
+    if rc != OK:
+        raise NovaAttnError(rc, "nova_attn_bwd_static_scratch")
 
 
 def nova_attn_poll_device_status(stream=None) -> int:

@@ -1,0 +1,73 @@
+"""nova_attn_bwd_static_scratch: the backward for callers that cannot allocate device memory.
+
+Such callers (code inside a fixed memory plan, plugins that only see their inputs and outputs, loops
+that must stay away from the allocator) cannot hand nova_attn_bwd a workspace, so this entry point
+keeps the dQ accumulator in an array built into the library.  The test calls it through the C ABI
+twice in a row on different inputs and checks each result against nova_attn_bwd on the same inputs:
+the second call must not be disturbed by what the first left in the shared array.  It also checks
+that no device memory is allocated by the call and that a problem too large for the array is refused.
+The file name sorts last so that a run stopping at the first failure has already run everything else.
+"""
+import pytest
+import torch
+
+from paper_2608_00029_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+
+def _forward_and_delta(na, cfg, seed, dev):
+    q, k, v, do = (x.to(dev) for x in W.make_inputs(cfg, seed=seed))
+    o = torch.empty_like(q)
+    lse = torch.empty((cfg.B, cfg.H, cfg.T), dtype=torch.float32, device=dev)
+    delta = torch.empty_like(lse)
+    na.nova_attn_fwd(q, k, v, o, lse, cfg.scale, cfg.causal)
+    na.nova_attn_bwd_preprocess(o, do, delta)
+    return q, k, v, o, do, lse, delta
+
+
+def test_static_scratch_backward_matches_workspace_backward_twice_in_a_row():
+    from paper_2608_00029_b200 import nova_attn as na
+    dev = torch.device("cuda:0")
+    torch.cuda.set_device(dev)
+    assert na.nova_attn_static_scratch_bytes() == 32 << 20
+    # two different problems, the second smaller than the first, so the second call meets an array
+    # full of the first call's partial sums
+    cases = [(W.CONFIGS["gpt2_small"].replace(B=2, H=3), 11), (W.AttnConfig("b", B=1, H=2, T=333, D=128, seed=0), 12)]
+    prepared = [(_forward_and_delta(na, cfg, seed, dev), cfg) for cfg, seed in cases]
+    want = []
+    for (q, k, v, o, do, lse, delta), cfg in prepared:
+        dq, dk, dv = (torch.empty_like(q) for _ in range(3))
+        na.nova_attn_bwd(q, k, v, o, do, lse, delta, dq, dk, dv, cfg.scale, cfg.causal)
+        want.append((dq, dk, dv))
+    outs = [tuple(torch.full_like(p[0][0], 5.0) for _ in range(3)) for p in prepared]
+    torch.cuda.synchronize()
+    before = torch.cuda.memory_allocated(dev)
+    for ((q, k, v, o, do, lse, delta), cfg), (dq, dk, dv) in zip(prepared, outs):   # back to back, no sync between
+        na.nova_attn_bwd_static_scratch(q, k, v, o, do, lse, delta, dq, dk, dv, cfg.scale, cfg.causal)
+    na.nova_attn_poll_device_status()
+    assert torch.cuda.memory_allocated(dev) == before
+    for (dq, dk, dv), (rq, rk, rv) in zip(outs, want):
+        # dK and dV do not touch the accumulator and are deterministic: identical bits
+        assert torch.equal(dk, rk) and torch.equal(dv, rv)
+        # dQ is summed with floating-point atomics in both variants: same bound as the parity tests
+        err = (dq.float() - rq.float()).abs()
+        assert torch.isfinite(dq.float()).all()
+        assert (err <= 2e-2 + 2e-2 * rq.float().abs()).all(), f"dQ differs by {float(err.max()):.3e}"
+        assert float(err.max()) <= 1e-2 * float(rq.float().abs().max()) + 1e-6
+
+
+def test_static_scratch_refuses_problems_larger_than_the_array():
+    from paper_2608_00029_b200 import nova_attn as na
+    dev = torch.device("cuda:0")
+    cfg = W.AttnConfig("big", B=3, H=12, T=4096, D=64, seed=0)      # 9.4 Mi elements > 8 Mi
+    assert na.nova_attn_bwd_workspace_bytes(cfg.B, cfg.H, cfg.T, cfg.D) > na.nova_attn_static_scratch_bytes()
+    shape = (cfg.B, cfg.H, cfg.T, cfg.D)
+    x = torch.zeros(shape, dtype=torch.bfloat16, device=dev)
+    r = torch.zeros(shape[:3], dtype=torch.float32, device=dev)
+    outs = [torch.full(shape, 3.0, dtype=torch.bfloat16, device=dev) for _ in range(3)]
+    with pytest.raises(na.NovaAttnError) as ei:
+        na.nova_attn_bwd_static_scratch(x, x, x, x, x, r, r, *outs, cfg.scale, True)
+    assert ei.value.status == na.ERR_WORKSPACE
+    torch.cuda.synchronize()
+    assert all(bool((o == 3.0).all()) for o in outs), "a refused call must not launch anything"
