@@ -88,8 +88,8 @@ int nova_attn_bwd_preprocess_exact(const void* Q, const void* K, const void* V, 
                                    float scale, int causal, void* stream);
 
 /*
- * Bytes of scratch nova_attn_bwd needs: an fp32 accumulator for dQ, [B,H,T,D].
- * Returns 0 if the shape is invalid.
+ * Bytes of scratch nova_attn_bwd needs: an fp32 accumulator for dQ, [B,H,T,D] (rounded up to
+ * 256 bytes).  Returns 0 if the shape is invalid.
  */
 size_t nova_attn_bwd_workspace_bytes(int B, int H, int T, int D);
 
@@ -104,7 +104,8 @@ size_t nova_attn_bwd_workspace_bytes(int B, int H, int T, int D);
  *   workspace   : device scratch of at least nova_attn_bwd_workspace_bytes(B,H,T,D) bytes, 16-byte
  *                 aligned; zeroed by the call itself on `stream`; contents afterwards unspecified.
  * dQ is accumulated in fp32 across key tiles with floating-point atomics, so its low-order bits may
- * differ from run to run; dK and dV are deterministic.
+ * differ from run to run; dK and dV are deterministic.  A final pass scales the accumulator, rounds it
+ * once to bf16 and writes dQ.
  */
 int nova_attn_bwd(const void* Q, const void* K, const void* V, const void* O, const void* dO,
                   const float* LSE, const float* Delta, void* dQ, void* dK, void* dV,

@@ -82,7 +82,7 @@ int device_state(DeviceState** out) {
 // call to a lookup when the same buffers are used step after step.
 struct MapKey {
     const void* ptr;
-    int D, T, BH, dev;
+    int D, T, BH, dev, elem_bytes;
 };
 struct MapEntry {
     MapKey key{};
@@ -92,33 +92,41 @@ struct MapEntry {
 constexpr int kMapCache = 128;
 MapEntry g_maps[kMapCache];
 
-int get_tensor_map(const void* ptr, int D, long long T, long long BH, CUtensorMap* out) {
+// elem_bytes 2: bf16 tensor, box [64, 128, 1]; elem_bytes 4: fp32 tensor, box [32, 128, 1].
+int get_tensor_map(const void* ptr, int D, long long T, long long BH, CUtensorMap* out, int elem_bytes = 2) {
     int dev = 0;
     cudaGetDevice(&dev);
-    const MapKey key{ptr, D, static_cast<int>(T), static_cast<int>(BH), dev};
+    const MapKey key{ptr, D, static_cast<int>(T), static_cast<int>(BH), dev, elem_bytes};
     const uint64_t h = (reinterpret_cast<uint64_t>(ptr) >> 8) * 0x9E3779B97F4A7C15ull + uint64_t(T) * 31 + uint64_t(BH) * 131 + D;
     std::lock_guard<std::mutex> lock(g_mutex);
     MapEntry& e = g_maps[(h >> 32) % kMapCache];
-    if (e.valid && std::memcmp(&e.key, &key, sizeof(MapKey)) == 0) {
+    if (e.valid && e.key.ptr == key.ptr && e.key.D == key.D && e.key.T == key.T && e.key.BH == key.BH &&
+        e.key.dev == key.dev && e.key.elem_bytes == key.elem_bytes) {
         *out = e.map;
         return NOVA_ATTN_OK;
     }
-    // [D, T, B*H] bf16, D contiguous; box [64, 128, 1]; rows past T read as zero.
+    // [D, T, B*H], D contiguous; 128-byte box rows; rows past T read as zero and are clipped on writes.
     const cuuint64_t dims[3] = {cuuint64_t(D), cuuint64_t(T), cuuint64_t(BH)};
-    const cuuint64_t strides[2] = {cuuint64_t(D) * 2, cuuint64_t(T) * cuuint64_t(D) * 2};
-    const cuuint32_t box[3] = {cuuint32_t(kBoxCols), cuuint32_t(kBlockQ), 1};
+    const cuuint64_t strides[2] = {cuuint64_t(D) * elem_bytes, cuuint64_t(T) * cuuint64_t(D) * elem_bytes};
+    const cuuint32_t box[3] = {cuuint32_t(128 / elem_bytes), cuuint32_t(kBlockQ), 1};
     const cuuint32_t estr[3] = {1, 1, 1};
     CUtensorMap m;
-    const CUresult r = g_encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box,
+    const CUresult r = g_encode(&m, elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32,
+                                3, const_cast<void*>(ptr), dims, strides, box,
                                 estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return fail_cuda(static_cast<int>(r));
-    std::memset(&e.key, 0, sizeof(MapKey));
     e.key = key;
     e.map = m;
     e.valid = true;
     *out = m;
     return NOVA_ATTN_OK;
+}
+
+// Workspace of the backward: the fp32 dQ accumulator [B,H,T,D], rounded up to 256 bytes.
+size_t acc_bytes(int B, int H, int T, int D) {
+    const size_t n = static_cast<size_t>(B) * H * T * D * sizeof(float);
+    return (n + 255) & ~size_t(255);
 }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -195,7 +203,7 @@ int nova_attn_bwd_preprocess_exact(const void* Q, const void* K, const void* V, 
 
 size_t nova_attn_bwd_workspace_bytes(int B, int H, int T, int D) {
     if (check_shape(B, H, T, D) != NOVA_ATTN_OK) return 0;
-    return static_cast<size_t>(B) * H * T * D * sizeof(float);
+    return acc_bytes(B, H, T, D);
 }
 
 int nova_attn_bwd_steps(const void* Q, const void* K, const void* V, const void* O, const void* dO, const float* LSE,
@@ -222,19 +230,20 @@ int nova_attn_bwd_steps(const void* Q, const void* K, const void* V, const void*
         if (e != cudaSuccess) return fail_cuda(e);
     }
     if (steps & NOVA_ATTN_BWD_STEP_MAIN) {
-        CUtensorMap tmQ, tmK, tmV, tmdO;
+        CUtensorMap tmQ, tmK, tmV, tmdO, tmAcc;
         if (int rc = get_tensor_map(Q, D, T, BH, &tmQ)) return rc;
         if (int rc = get_tensor_map(K, D, T, BH, &tmK)) return rc;
         if (int rc = get_tensor_map(V, D, T, BH, &tmV)) return rc;
         if (int rc = get_tensor_map(dO, D, T, BH, &tmdO)) return rc;
+        if (int rc = get_tensor_map(acc, D, T, BH, &tmAcc, 4)) return rc;
         const AttnShape s{B, H, T, D, causal != 0, scale};
-        e = launch_attn_bwd(tmQ, tmK, tmV, tmdO, LSE, Delta, acc, static_cast<__nv_bfloat16*>(dK),
+        e = launch_attn_bwd(tmQ, tmK, tmV, tmdO, tmAcc, LSE, Delta, acc, static_cast<__nv_bfloat16*>(dK),
                             static_cast<__nv_bfloat16*>(dV), s, st->dev_status, cs);
         if (e != cudaSuccess) return fail_cuda(e);
     }
     if (steps & NOVA_ATTN_BWD_STEP_CONVERT) {
-        e = launch_dq_convert(acc, static_cast<__nv_bfloat16*>(dQ), static_cast<long long>(need / sizeof(float)),
-                              scale, st->num_sms, cs);
+        e = launch_dq_convert(acc, static_cast<__nv_bfloat16*>(dQ), static_cast<long long>(B) * H * T * D, scale,
+                              st->num_sms, cs);
         if (e != cudaSuccess) return fail_cuda(e);
     }
     return NOVA_ATTN_OK;

@@ -34,11 +34,11 @@ cudaError_t launch_attn_delta(const CUtensorMap& tmQ, const CUtensorMap& tmK, co
                               int* dev_status, cudaStream_t stream);
 cudaError_t configure_attn_delta();
 
-// Backward main kernel: accumulates unscaled dQ into `dq_acc` (fp32 [B,H,T,D], zeroed beforehand),
-// writes dK and dV.
+// Backward main kernel: adds unscaled dQ partial tiles into `dq_acc` (fp32 [B,H,T,D], zero on entry; also
+// described by `tmAcc`: fp32 [D, T, B*H], box [32, 128, 1], 128-byte swizzle) and writes dK and dV.
 cudaError_t launch_attn_bwd(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV,
-                            const CUtensorMap& tmdO, const float* LSE, const float* Delta, float* dq_acc,
-                            __nv_bfloat16* dK, __nv_bfloat16* dV, const AttnShape& s, int* dev_status,
+                            const CUtensorMap& tmdO, const CUtensorMap& tmAcc, const float* LSE, const float* Delta,
+                            float* dq_acc, __nv_bfloat16* dK, __nv_bfloat16* dV, const AttnShape& s, int* dev_status,
                             cudaStream_t stream);
 cudaError_t configure_attn_bwd();
 

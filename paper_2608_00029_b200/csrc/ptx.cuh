@@ -7,6 +7,9 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
+#ifdef NOVA_EXP_TRACE
+#include <cstdio>
+#endif
 
 namespace nova {
 
@@ -60,6 +63,10 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
             if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag != 0) return false;
         if (clock64() - t0 > kWaitLimitCycles) {
+#ifdef NOVA_EXP_TRACE
+            if (*abort_flag == 0)
+                printf("TIMEOUT block %d thread %d bar 0x%x parity %u\n", blockIdx.x, threadIdx.x, smem_u32(bar), parity);
+#endif
             *abort_flag = 1;
             return false;
         }
@@ -78,6 +85,13 @@ __device__ __forceinline__ void tma_load_3d(void* smem_dst, const CUtensorMap* m
         "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
         ::"r"(smem_u32(smem_dst)), "l"(m), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2)
         : "memory");
+}
+// 3-D tiled reduce-add shared (this CTA) -> global through a tensor map: global += smem box.
+// Completion is tracked by this thread's bulk async-groups.  Coordinates must be non-negative.
+__device__ __forceinline__ void tma_reduce_add_3d(const CUtensorMap* m, const void* smem_src, int c0, int c1, int c2) {
+    asm volatile("cp.reduce.async.bulk.tensor.3d.global.shared::cta.add.bulk_group [%0, {%2, %3, %4}], [%1];" ::"l"(m),
+                 "r"(smem_u32(smem_src)), "r"(c0), "r"(c1), "r"(c2)
+                 : "memory");
 }
 // Make generic-proxy writes to shared memory visible to the async proxy (TMA, UMMA operand reads).
 __device__ __forceinline__ void fence_proxy_async_smem() {
@@ -219,6 +233,23 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 __device__ __forceinline__ void red_add_v4_f32(float* addr, float a, float b, float c, float d) {
     asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(a), "f"(b), "f"(c), "f"(d)
                  : "memory");
+}
+// Bulk asynchronous reduction shared -> global: global[i] += smem[i] for `bytes`/4 floats, performed
+// by the copy engine at L2.  Both addresses 16-byte aligned, `bytes` a multiple of 16.
+__device__ __forceinline__ void bulk_reduce_add_f32(float* gdst, const void* smem_src, uint32_t bytes) {
+    asm volatile("cp.reduce.async.bulk.global.shared::cta.bulk_group.add.f32 [%0], [%1], %2;" ::"l"(gdst),
+                 "r"(smem_u32(smem_src)), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_commit_group() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// At most N of this thread's bulk groups still pending (.read: only their shared-memory reads).
+template <int N>
+__device__ __forceinline__ void bulk_wait_group() {
+    asm volatile("cp.async.bulk.wait_group %0;" ::"n"(N) : "memory");
+}
+template <int N>
+__device__ __forceinline__ void bulk_wait_group_read() {
+    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
 }
 __device__ __forceinline__ void named_barrier_sync(int id, int nthreads) {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");

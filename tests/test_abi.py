@@ -43,6 +43,7 @@ def test_workspace_query(lib):
     from paper_2608_00029_b200 import nova_attn as na
     assert na.nova_attn_bwd_workspace_bytes(8, 12, 1024, 64) == 8 * 12 * 1024 * 64 * 4
     assert na.nova_attn_bwd_workspace_bytes(2, 12, 8192, 128) == 2 * 12 * 8192 * 128 * 4
+    assert na.nova_attn_bwd_workspace_bytes(1, 1, 1, 64) == 256
     assert na.nova_attn_bwd_workspace_bytes(1, 1, 1, 96) == 0      # unsupported head dim
     assert na.nova_attn_bwd_workspace_bytes(0, 1, 1, 64) == 0
 
