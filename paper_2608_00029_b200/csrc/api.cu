@@ -230,15 +230,17 @@ int nova_attn_bwd_steps(const void* Q, const void* K, const void* V, const void*
         if (e != cudaSuccess) return fail_cuda(e);
     }
     if (steps & NOVA_ATTN_BWD_STEP_MAIN) {
-        CUtensorMap tmQ, tmK, tmV, tmdO, tmAcc;
+        CUtensorMap tmQ, tmK, tmV, tmdO, tmAcc, tmdK, tmdV;
         if (int rc = get_tensor_map(Q, D, T, BH, &tmQ)) return rc;
         if (int rc = get_tensor_map(K, D, T, BH, &tmK)) return rc;
         if (int rc = get_tensor_map(V, D, T, BH, &tmV)) return rc;
         if (int rc = get_tensor_map(dO, D, T, BH, &tmdO)) return rc;
         if (int rc = get_tensor_map(acc, D, T, BH, &tmAcc, 4)) return rc;
+        if (int rc = get_tensor_map(dK, D, T, BH, &tmdK)) return rc;
+        if (int rc = get_tensor_map(dV, D, T, BH, &tmdV)) return rc;
         const AttnShape s{B, H, T, D, causal != 0, scale};
-        e = launch_attn_bwd(tmQ, tmK, tmV, tmdO, tmAcc, LSE, Delta, acc, static_cast<__nv_bfloat16*>(dK),
-                            static_cast<__nv_bfloat16*>(dV), s, st->dev_status, cs);
+        e = launch_attn_bwd(tmQ, tmK, tmV, tmdO, tmAcc, tmdK, tmdV, LSE, Delta, acc, static_cast<__nv_bfloat16*>(dK),
+                            static_cast<__nv_bfloat16*>(dV), s, st->num_sms, st->dev_status, cs);
         if (e != cudaSuccess) return fail_cuda(e);
     }
     if (steps & NOVA_ATTN_BWD_STEP_CONVERT) {

@@ -7,9 +7,6 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
-#ifdef NOVA_EXP_TRACE
-#include <cstdio>
-#endif
 
 namespace nova {
 
@@ -51,6 +48,21 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     return ok != 0;
 }
 
+// Same test, but the hardware may keep the thread suspended for up to `hint_ns` while the phase is
+// incomplete (it resumes at once when the phase completes).  A suspended thread issues nothing, so
+// waiting warps do not take issue slots from the warps that share their scheduler.
+__device__ __forceinline__ bool mbar_try_wait_suspend(uint64_t* bar, uint32_t parity, uint32_t hint_ns) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity), "r"(hint_ns)
+        : "memory");
+    return ok != 0;
+}
+
 // Bounded wait.  Returns false if the phase did not complete within kWaitLimitCycles or if another
 // thread of the CTA already gave up (*abort_flag != 0); the caller then leaves through the common
 // exit path.  `abort_flag` lives in shared memory.
@@ -59,14 +71,10 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
     const long long t0 = clock64();
     for (;;) {
 #pragma unroll 1
-        for (int i = 0; i < 32; ++i)
-            if (mbar_try_wait(bar, parity)) return true;
+        for (int i = 0; i < 8; ++i)
+            if (mbar_try_wait_suspend(bar, parity, 20000u)) return true;
         if (*abort_flag != 0) return false;
         if (clock64() - t0 > kWaitLimitCycles) {
-#ifdef NOVA_EXP_TRACE
-            if (*abort_flag == 0)
-                printf("TIMEOUT block %d thread %d bar 0x%x parity %u\n", blockIdx.x, threadIdx.x, smem_u32(bar), parity);
-#endif
             *abort_flag = 1;
             return false;
         }
@@ -90,6 +98,13 @@ __device__ __forceinline__ void tma_load_3d(void* smem_dst, const CUtensorMap* m
 // Completion is tracked by this thread's bulk async-groups.  Coordinates must be non-negative.
 __device__ __forceinline__ void tma_reduce_add_3d(const CUtensorMap* m, const void* smem_src, int c0, int c1, int c2) {
     asm volatile("cp.reduce.async.bulk.tensor.3d.global.shared::cta.add.bulk_group [%0, {%2, %3, %4}], [%1];" ::"l"(m),
+                 "r"(smem_u32(smem_src)), "r"(c0), "r"(c1), "r"(c2)
+                 : "memory");
+}
+// 3-D tiled store shared (this CTA) -> global through a tensor map; rows outside the tensor are
+// clipped.  Completion is tracked by this thread's bulk async-groups.
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* m, const void* smem_src, int c0, int c1, int c2) {
+    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];" ::"l"(m),
                  "r"(smem_u32(smem_src)), "r"(c0), "r"(c1), "r"(c2)
                  : "memory");
 }
@@ -167,6 +182,18 @@ __device__ __forceinline__ uint64_t umma_smem_desc_sw128(uint32_t smem_addr, uin
     d |= uint64_t(1) << 46;   // descriptor version for sm_100
     d |= uint64_t(2) << 61;   // SWIZZLE_128B
     return d;
+}
+
+// The same descriptor split in two: the constant upper word and the lower word as a function of the
+// address, so that a hot loop only adds a byte offset (>> 4) to a precomputed lower word.
+__device__ __forceinline__ uint32_t umma_desc_hi_sw128(uint32_t sbo_bytes) {
+    return ((sbo_bytes >> 4) & 0x3FFFu) | (1u << 14) | (2u << 29);
+}
+__device__ __forceinline__ uint32_t umma_desc_lo(uint32_t smem_addr, uint32_t lbo_bytes) {
+    return ((smem_addr & 0x3FFFFu) >> 4) | (((lbo_bytes >> 4) & 0x3FFFu) << 16);
+}
+__device__ __forceinline__ uint64_t umma_desc_join(uint32_t lo, uint32_t hi) {
+    return (static_cast<uint64_t>(hi) << 32) | lo;
 }
 
 // TMEM address: lane in bits [31:16], column in bits [15:0].

@@ -127,13 +127,16 @@ def test_edge_shapes(B, H, T, D, causal):
 
 
 def test_peaked_softmax_large_scores():
-    """Scores ~ N(0, 64): exercises the running-max rescale and the exp range."""
+    """Scores ~ N(0, 16^2) (Q, K ~ 4 N(0,1)): exercises the running-max rescale and the exp range far
+    beyond the five configurations.  |K| and |dS| are 4x and ~10x larger than there, and dQ, dK are sums
+    of a few large bf16-rounded terms dS*K, so the gradients are held to three times the usual bound
+    (forward results to the usual one)."""
     h = _harness()
     cfg = W.AttnConfig("peaked", B=1, H=4, T=512, D=64, seed=77, qk_factor=4.0)
     Q, K, V, dO = W.make_inputs(cfg)
     got = h.run_gpu(Q, K, V, dO, cfg.scale, True, exact_delta=True)
     ref = h.run_oracle(Q, K, V, dO, cfg.scale, True)
-    h.compare(h.select_heads(got, None), ref, label="peaked: ", dO=ref["dO_in"])
+    h.compare(h.select_heads(got, None), ref, label="peaked: ", dO=ref["dO_in"], bwd_factor=3.0)
 
 
 def test_increasing_scores_force_rescales():
