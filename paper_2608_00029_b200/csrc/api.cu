@@ -157,12 +157,13 @@ int nova_attn_fwd(const void* Q, const void* K, const void* V, void* O, float* L
     DeviceState* st = nullptr;
     if (int rc = device_state(&st)) return rc;
     const long long BH = static_cast<long long>(B) * H;
-    CUtensorMap tmQ, tmK, tmV;
+    CUtensorMap tmQ, tmK, tmV, tmO;
     if (int rc = get_tensor_map(Q, D, T, BH, &tmQ)) return rc;
     if (int rc = get_tensor_map(K, D, T, BH, &tmK)) return rc;
     if (int rc = get_tensor_map(V, D, T, BH, &tmV)) return rc;
+    if (int rc = get_tensor_map(O, D, T, BH, &tmO)) return rc;
     const AttnShape s{B, H, T, D, causal != 0, scale};
-    const cudaError_t e = launch_attn_fwd(tmQ, tmK, tmV, static_cast<__nv_bfloat16*>(O), LSE, s, st->dev_status,
+    const cudaError_t e = launch_attn_fwd(tmQ, tmK, tmV, tmO, LSE, s, st->num_sms, st->dev_status,
                                           static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? NOVA_ATTN_OK : fail_cuda(e);
 }

@@ -1,133 +1,233 @@
 // Fused causal attention forward for sm_100a (paper Section 4.2: score contraction, index mask,
 // base-2 online softmax, value contraction, causal loop clamp, 1/sum epilogue, LSE saved).
 //
-// One CTA owns one 128-row query tile of one (batch, head) and walks the key tiles up to the
-// diagonal.  Roles:
-//   warp 0      TMA producer: Q once, then K and V tiles through mbarrier-guarded rings
-//   warp 1      UMMA issuer:  S = Q K^T  (operands in shared memory, accumulator in TMEM)
-//                             O += P V   (P read from TMEM as bf16, V from shared memory)
-//   warps 2..5  softmax: one thread per query row reads its S row from TMEM, keeps the running
-//               max / sum in registers, writes bf16 P back over S, rescales O in TMEM only when the
-//               row maximum has grown by more than 2^8 (exact: the final 1/sum and the LSE use the
-//               same reference maximum), and runs the epilogue.
-// TMEM: columns [0,128) hold S (fp32) then P (bf16 pairs in [0,64)); [128,128+D) hold O (fp32).
-// Two CTAs are resident per SM, so one CTA's softmax overlaps the other's tensor-core work.
+// A work item is a block of 256 query rows of one (batch, head): two 128-row query tiles, A and B,
+// that share every K/V tile they both need.  The kernel is persistent: one CTA per SM walks a fixed
+// list of items, heaviest first (the last query block of a causal problem sees every key tile),
+// dealt out in zig-zag order.  Roles (384 threads):
+//   warp 0       TMA producer: Q tiles per item, K and V tiles through mbarrier-guarded rings
+//   warp 1       UMMA issuer:  S_t = Q_t K^T  (operands in shared memory, accumulator in TMEM)
+//                              O_t += P_t V   (P read from TMEM as bf16, V from shared memory)
+//                interleaved over the two tiles: while the softmax warps of tile A work on key tile
+//                j+1 the tensor core runs P V and the next Q K^T of tile B, and vice versa
+//   warps 4-7    softmax of tile A, warps 8-11 softmax of tile B: one thread per query row reads its
+//                S row from TMEM, keeps the running max / sum in registers, writes bf16 P back over
+//                S, rescales O in TMEM only when the row maximum has grown by more than 2^8 (exact:
+//                the final 1/sum and the LSE use the same reference maximum), and at the end of the
+//                item normalises O, stages it in the (now idle) Q tile buffer and sends it out with
+//                TMA stores.
+// TMEM columns: S_A [0,128)  S_B [128,256)  O_A [256,256+D)  O_B [256+D,256+2D); P_t is bf16 pairs
+// over the first 64 columns of S_t.
+//
+// Warp-wide .sync.aligned instructions (TMEM loads/stores) need the whole warp together: wherever
+// one lane does extra work (the store leader), the warp is rejoined with a vote before the next one.
 #include "kernels.h"
 #include "ptx.cuh"
 
 namespace nova {
 namespace {
 
-constexpr int kFwdThreads = 192;
-constexpr int kFwdTmemCols = 256;
-constexpr int kColS = 0;
-constexpr int kColO = 128;
+constexpr int kFwdThreads = 384;
+constexpr int kFwdTmemCols = 512;
 constexpr float kRescaleThreshold = 8.0f;  // log2 units
+constexpr int kBlockRows = 2 * kBlockQ;    // query rows per work item
 
 template <int D>
 struct FwdCfg {
     static constexpr int kHalves = D / kBoxCols;
     static constexpr int kTileBytes = kHalves * kHalfTileBytes;
-    static constexpr int kStages = (D == 64) ? 2 : 1;
-    static constexpr int kOffQ = 0;
-    static constexpr int kOffK = kTileBytes;
-    static constexpr int kOffV = kTileBytes * (1 + kStages);
-    static constexpr int kOffBar = kTileBytes * (1 + 2 * kStages);
-    static constexpr int kSmemBytes = kOffBar + 256 + 1024;  // + barriers + alignment slack
+    static constexpr int kQStages = (D == 64) ? 2 : 1;
+    static constexpr int kKVStages = 2;
+    static constexpr int kOffQ = 0;                                    // [kQStages][2 tiles]
+    static constexpr int kOffK = kQStages * 2 * kTileBytes;            // [kKVStages]
+    static constexpr int kOffV = kOffK + kKVStages * kTileBytes;       // [kKVStages]
+    static constexpr int kOffBar = kOffV + kKVStages * kTileBytes;
+    static constexpr int kSmemBytes = kOffBar + 512 + 1024;
+    static constexpr int kColS = 0;      // + 128 * tile
+    static constexpr int kColO = 256;    // + D * tile
 };
 
 struct FwdBars {
-    uint64_t q_full;
+    uint64_t q_full[2], q_empty[2];
     uint64_t k_full[2], k_empty[2], v_full[2], v_empty[2];
-    uint64_t s_full, p_ready, pv_done, drain;
+    uint64_t s_full[2], p_ready[2], pv_done[2], o_free[2], o_staged[2];  // per query tile
+    uint64_t drain;
     uint32_t tmem_base;
     int abort_flag;
 };
 
+// This CTA's list of work items: 256-row query blocks, heaviest first, dealt in zig-zag passes.
+struct FwdWork {
+    int n_items, n_ctas, cta, BH, n_blocks, n_kv_all, T;
+    bool causal;
+    __device__ __forceinline__ int passes() const { return (n_items + n_ctas - 1) / n_ctas; }
+    // Item of pass p: block index, head, and the number of key tiles each query tile visits
+    // (0 if the tile lies entirely past the end of the sequence).
+    __device__ __forceinline__ bool get(int p, int* blk, int* bh, int* n_a, int* n_b) const {
+        const int idx = p * n_ctas + ((p & 1) ? (n_ctas - 1 - cta) : cta);
+        if (idx >= n_items) return false;
+        *blk = n_blocks - 1 - idx / BH;
+        *bh = idx % BH;
+        const int qt_a = 2 * (*blk), qt_b = qt_a + 1;
+        // causal clamp of the key loop: tile qt visits key tiles 0..qt
+        *n_a = causal ? min(qt_a + 1, n_kv_all) : n_kv_all;
+        *n_b = (qt_b * kBlockQ < T) ? (causal ? min(qt_b + 1, n_kv_all) : n_kv_all) : 0;
+        return true;
+    }
+};
+
 template <int D>
 __device__ __forceinline__ void fwd_producer(const CUtensorMap* tmQ, const CUtensorMap* tmK,
-                                             const CUtensorMap* tmV, uint8_t* smem, FwdBars* bars, int qt, int bh,
-                                             int n_kv) {
+                                             const CUtensorMap* tmV, uint8_t* smem, FwdBars* bars,
+                                             const FwdWork& wk) {
     using Cfg = FwdCfg<D>;
     volatile int* abort_flag = &bars->abort_flag;
-    int armed_k[2] = {-1, -1}, armed_v[2] = {-1, -1};
-    mbar_expect_tx(&bars->q_full, Cfg::kTileBytes);
-#pragma unroll
-    for (int h = 0; h < Cfg::kHalves; ++h)
-        tma_load_3d(smem + Cfg::kOffQ + h * kHalfTileBytes, tmQ, &bars->q_full, h * kBoxCols, qt * kBlockQ, bh);
+    int armed_q[2] = {-1, -1}, armed_k[2] = {-1, -1}, armed_v[2] = {-1, -1};
     bool ok = true;
-    for (int j = 0; j < n_kv && ok; ++j) {
-        const int st = j % Cfg::kStages;
-        const uint32_t ph = (j / Cfg::kStages) & 1;
-        ok = mbar_wait(&bars->k_empty[st], ph ^ 1, abort_flag);
+    int w = 0, g = 0;  // items and key tiles loaded so far
+    for (int p = 0; p < wk.passes() && ok; ++p) {
+        int blk, bh, n_a, n_b;
+        if (!wk.get(p, &blk, &bh, &n_a, &n_b)) continue;
+        const int qs = w % Cfg::kQStages;
+        const uint32_t qph = (w / Cfg::kQStages) & 1;
+        ok = mbar_wait(&bars->q_empty[qs], qph ^ 1, abort_flag);
         if (!ok) break;
-        mbar_expect_tx(&bars->k_full[st], Cfg::kTileBytes);
-        armed_k[st] = ph;
+        mbar_expect_tx(&bars->q_full[qs], 2 * Cfg::kTileBytes);  // rows past T arrive as zeros
+        armed_q[qs] = qph;
 #pragma unroll
-        for (int h = 0; h < Cfg::kHalves; ++h)
-            tma_load_3d(smem + Cfg::kOffK + st * Cfg::kTileBytes + h * kHalfTileBytes, tmK, &bars->k_full[st],
-                        h * kBoxCols, j * kBlockK, bh);
-        ok = mbar_wait(&bars->v_empty[st], ph ^ 1, abort_flag);
-        if (!ok) break;
-        mbar_expect_tx(&bars->v_full[st], Cfg::kTileBytes);
-        armed_v[st] = ph;
+        for (int t = 0; t < 2; ++t)
 #pragma unroll
-        for (int h = 0; h < Cfg::kHalves; ++h)
-            tma_load_3d(smem + Cfg::kOffV + st * Cfg::kTileBytes + h * kHalfTileBytes, tmV, &bars->v_full[st],
-                        h * kBoxCols, j * kBlockK, bh);
+            for (int h = 0; h < Cfg::kHalves; ++h)
+                tma_load_3d(smem + Cfg::kOffQ + (qs * 2 + t) * Cfg::kTileBytes + h * kHalfTileBytes, tmQ,
+                            &bars->q_full[qs], h * kBoxCols, blk * kBlockRows + t * kBlockQ, bh);
+        const int n = max(n_a, n_b);
+        for (int j = 0; j < n; ++j, ++g) {
+            const int st = g & 1;
+            const uint32_t ph = (g >> 1) & 1;
+            ok = mbar_wait(&bars->k_empty[st], ph ^ 1, abort_flag);
+            if (!ok) break;
+            mbar_expect_tx(&bars->k_full[st], Cfg::kTileBytes);
+            armed_k[st] = ph;
+#pragma unroll
+            for (int h = 0; h < Cfg::kHalves; ++h)
+                tma_load_3d(smem + Cfg::kOffK + st * Cfg::kTileBytes + h * kHalfTileBytes, tmK, &bars->k_full[st],
+                            h * kBoxCols, j * kBlockK, bh);
+            ok = mbar_wait(&bars->v_empty[st], ph ^ 1, abort_flag);
+            if (!ok) break;
+            mbar_expect_tx(&bars->v_full[st], Cfg::kTileBytes);
+            armed_v[st] = ph;
+#pragma unroll
+            for (int h = 0; h < Cfg::kHalves; ++h)
+                tma_load_3d(smem + Cfg::kOffV + st * Cfg::kTileBytes + h * kHalfTileBytes, tmV, &bars->v_full[st],
+                            h * kBoxCols, j * kBlockK, bh);
+        }
+        ++w;
     }
     if (!ok) {
-        // Giving up: let the copies already in flight land before the CTA (and its shared memory) goes away.
+        // Giving up: let the copies already in flight land before the CTA's shared memory goes away.
         int none = 0;
-        (void)mbar_wait(&bars->q_full, 0, &none);
-        for (int st = 0; st < Cfg::kStages; ++st) {
-            if (armed_k[st] >= 0) (void)mbar_wait(&bars->k_full[st], armed_k[st], &none);
-            if (armed_v[st] >= 0) (void)mbar_wait(&bars->v_full[st], armed_v[st], &none);
+        for (int s = 0; s < 2; ++s) {
+            if (armed_q[s] >= 0) (void)mbar_wait(&bars->q_full[s], armed_q[s], &none);
+            if (armed_k[s] >= 0) (void)mbar_wait(&bars->k_full[s], armed_k[s], &none);
+            if (armed_v[s] >= 0) (void)mbar_wait(&bars->v_full[s], armed_v[s], &none);
         }
     }
 }
 
 template <int D>
-__device__ __forceinline__ void fwd_mma(uint8_t* smem, FwdBars* bars, uint32_t tmem_base, int n_kv) {
+__device__ __forceinline__ void fwd_mma(uint8_t* smem, FwdBars* bars, uint32_t tmem_base, const FwdWork& wk) {
     using Cfg = FwdCfg<D>;
     volatile int* abort_flag = &bars->abort_flag;
     constexpr uint32_t kIdescQK = umma_idesc_bf16(128, 128, 0, 0);
     constexpr uint32_t kIdescPV = umma_idesc_bf16(128, D, 0, 1);
-    const uint32_t sQ = smem_u32(smem + Cfg::kOffQ);
-    const uint32_t t_s = tmem_base + kColS;
-    const uint32_t t_o = tmem_base + kColO;
-    bool ok = mbar_wait(&bars->q_full, 0, abort_flag);
-    for (int j = 0; j < n_kv && ok; ++j) {
-        const int st = j % Cfg::kStages;
-        const uint32_t ph = (j / Cfg::kStages) & 1;
-        ok = mbar_wait(&bars->k_full[st], ph, abort_flag);
-        if (!ok) break;
-        tc_fence_after();
-        const uint32_t sK = smem_u32(smem + Cfg::kOffK + st * Cfg::kTileBytes);
-        // S = Q K^T: both operands K-major; 16 head-dim elements (32 bytes) per instruction.
+    const uint32_t hi = umma_desc_hi_sw128(1024);
+    // Descriptor lower words per buffer; in the loops only a constant (byte offset >> 4) is added.
+    uint32_t k_k[2], v_m[2];
+#pragma unroll
+    for (int st = 0; st < 2; ++st) {
+        k_k[st] = umma_desc_lo(smem_u32(smem + Cfg::kOffK + st * Cfg::kTileBytes), 16);
+        v_m[st] = umma_desc_lo(smem_u32(smem + Cfg::kOffV + st * Cfg::kTileBytes), kHalfTileBytes);
+    }
+    uint32_t q_k[2] = {0, 0};  // per item: the two query tiles
+    bool ok = true;
+    int w = 0, g = 0;
+    int c[2] = {0, 0};   // key tiles processed so far per query tile (phases of its barriers)
+    int wt[2] = {0, 0};  // items in which the query tile took part so far (phases of o_free)
+
+    // S_t = Q_t K^T for the key tile in stage gk & 1: both operands K-major, 16 head-dim elements
+    // (32 bytes) per instruction.
+    auto issue_qk = [&](int t, int gk) {
+        const uint32_t t_s = tmem_base + Cfg::kColS + 128 * t;
+        const uint32_t b = k_k[gk & 1];
 #pragma unroll
         for (int k = 0; k < D / 16; ++k) {
-            const uint32_t off = (k / 4) * kHalfTileBytes + (k % 4) * 32;
-            umma_ss(t_s, umma_smem_desc_sw128(sQ + off, 16, 1024), umma_smem_desc_sw128(sK + off, 16, 1024),
-                    kIdescQK, k > 0 ? 1u : 0u);
+            const uint32_t off = ((k / 4) * kHalfTileBytes + (k % 4) * 32) >> 4;
+            umma_ss(t_s, umma_desc_join(q_k[t] + off, hi), umma_desc_join(b + off, hi), kIdescQK, k > 0 ? 1u : 0u);
         }
-        tc_commit(&bars->k_empty[st]);
-        tc_commit(&bars->s_full);
-        ok = mbar_wait(&bars->p_ready, j & 1, abort_flag);
-        if (!ok) break;
-        ok = mbar_wait(&bars->v_full[st], ph, abort_flag);
+        tc_commit(&bars->s_full[t]);
+    };
+
+    for (int p = 0; p < wk.passes() && ok; ++p) {
+        int blk, bh, n_a, n_b;
+        if (!wk.get(p, &blk, &bh, &n_a, &n_b)) continue;
+        const int n_t[2] = {n_a, n_b};
+        const int n = max(n_a, n_b);
+        const int qs = w % Cfg::kQStages;
+#pragma unroll
+        for (int t = 0; t < 2; ++t)
+            q_k[t] = umma_desc_lo(smem_u32(smem + Cfg::kOffQ + (qs * 2 + t) * Cfg::kTileBytes), 16);
+        ok = mbar_wait(&bars->q_full[qs], (w / Cfg::kQStages) & 1, abort_flag);
+        if (ok) ok = mbar_wait(&bars->k_full[g & 1], (g >> 1) & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
-        const uint32_t sV = smem_u32(smem + Cfg::kOffV + st * Cfg::kTileBytes);
-        // O += P V: P from TMEM (16 keys = 8 packed columns per instruction), V is MN-major
-        // (rows = keys, 64 head-dim elements per 128-byte row, second 64-wide half at +16 KB).
+        // The S columns of both tiles are free: their last P was consumed by a P V queued earlier.
+        if (n_a > 0) issue_qk(0, g);
+        if (n_b > 0) issue_qk(1, g);
+        tc_commit(&bars->k_empty[g & 1]);  // K tile 0 is no longer read once these have run
+        for (int j = 0; j < n && ok; ++j, ++g) {
+            const int st = g & 1;
+            bool next_k_ready = false;
 #pragma unroll
-        for (int k = 0; k < kBlockK / 16; ++k) {
-            umma_ts(t_o, t_s + k * 8, umma_smem_desc_sw128(sV + k * 2048, kHalfTileBytes, 1024), kIdescPV,
-                    (j > 0 || k > 0) ? 1u : 0u);
+            for (int t = 0; t < 2; ++t) {
+                if (j >= n_t[t]) continue;
+                const uint32_t t_s = tmem_base + Cfg::kColS + 128 * t;
+                const uint32_t t_o = tmem_base + Cfg::kColO + D * t;
+                ok = mbar_wait(&bars->p_ready[t], c[t] & 1, abort_flag);
+                if (!ok) break;
+                if (j == 0) {
+                    ok = mbar_wait(&bars->v_full[st], (g >> 1) & 1, abort_flag);
+                    // the previous item's O_t must have been read out of TMEM before it is overwritten
+                    if (ok && wt[t] > 0) ok = mbar_wait(&bars->o_free[t], (wt[t] - 1) & 1, abort_flag);
+                } else if (t == 0 || j >= n_t[0]) {
+                    ok = mbar_wait(&bars->v_full[st], (g >> 1) & 1, abort_flag);
+                }
+                if (!ok) break;
+                tc_fence_after();
+                // O_t += P_t V: P from TMEM (16 keys = 8 packed columns per instruction), V is MN-major
+                // (rows = keys, 64 head-dim elements per 128-byte row, second 64-wide half at +16 KB).
+#pragma unroll
+                for (int k = 0; k < kBlockK / 16; ++k)
+                    umma_ts(t_o, t_s + k * 8, umma_desc_join(v_m[st] + k * 128, hi), kIdescPV,
+                            (j > 0 || k > 0) ? 1u : 0u);
+                tc_commit(&bars->pv_done[t]);
+                ++c[t];
+                if (j + 1 < n_t[t]) {  // the S_t columns are free again once this P V has run
+                    if (!next_k_ready) {
+                        ok = mbar_wait(&bars->k_full[st ^ 1], ((g + 1) >> 1) & 1, abort_flag);
+                        if (!ok) break;
+                        tc_fence_after();
+                        next_k_ready = true;
+                    }
+                    issue_qk(t, g + 1);
+                }
+            }
+            if (!ok) break;
+            tc_commit(&bars->v_empty[st]);                    // V tile j is no longer read
+            if (j + 1 < n) tc_commit(&bars->k_empty[st ^ 1]);  // nor K tile j+1 (both Q K^T are queued)
         }
-        tc_commit(&bars->v_empty[st]);
-        tc_commit(&bars->pv_done);
+        if (n_a > 0) ++wt[0];
+        if (n_b > 0) ++wt[1];
+        ++w;
     }
     if (!ok) {
         // Drain whatever was issued before leaving so TMEM can be released safely.
@@ -138,156 +238,209 @@ __device__ __forceinline__ void fwd_mma(uint8_t* smem, FwdBars* bars, uint32_t t
 }
 
 template <int D, bool kCausal>
-__device__ __forceinline__ void fwd_softmax(FwdBars* bars, uint32_t tmem_base, __nv_bfloat16* O, float* LSE, int T,
-                                            int qt, int bh, int n_kv, float scale, int warp, int lane) {
+__device__ __forceinline__ void fwd_softmax(uint8_t* smem, FwdBars* bars, uint32_t tmem_base, const CUtensorMap* tmO,
+                                            float* __restrict__ LSE, float scale, const FwdWork& wk, int t, int swarp,
+                                            int lane) {
+    using Cfg = FwdCfg<D>;
     volatile int* abort_flag = &bars->abort_flag;
-    const uint32_t lane_base = 32u * (warp & 3);
+    const uint32_t lane_base = 32u * (swarp & 3);
     const int row_local = lane_base + lane;
-    const int row = qt * kBlockQ + row_local;
-    const uint32_t t_s = tmem_addr(tmem_base, lane_base, kColS);
-    const uint32_t t_o = tmem_addr(tmem_base, lane_base, kColO);
+    const bool leader = (swarp == 0 && lane == 0);
+    const uint32_t t_s = tmem_addr(tmem_base, lane_base, Cfg::kColS + 128 * t);
+    const uint32_t t_o = tmem_addr(tmem_base, lane_base, Cfg::kColO + D * t);
     const float c = scale * kLog2e;
-    float m_ref = -INFINITY;  // reference maximum of the raw (unscaled) scores
-    float l = 0.f;
+    const int T = wk.T;
     bool ok = true;
+    int w = 0, wt = 0, cnt = 0;  // items, items this tile took part in, key tiles processed by this tile
 
-    for (int j = 0; j < n_kv; ++j) {
-        ok = mbar_wait(&bars->s_full, j & 1, abort_flag);
-        if (!ok) break;
-        tc_fence_after();
-        uint32_t sr[128];
-        tmem_ld_x32(t_s + 0, sr + 0);
-        tmem_ld_x32(t_s + 32, sr + 32);
-        tmem_ld_x32(t_s + 64, sr + 64);
-        tmem_ld_x32(t_s + 96, sr + 96);
-        tmem_wait_ld();
-
-        // Mask from indices only: the diagonal tile keeps key <= query; a ragged last tile keeps key < T.
-        const bool diag = kCausal && (j == qt);
-        const int keys_left = T - j * kBlockK;
-        if (diag || keys_left < kBlockK) {
-            const int lim = diag ? min(row_local, keys_left - 1) : keys_left - 1;
-#pragma unroll
-            for (int i = 0; i < 128; ++i)
-                if (i > lim) sr[i] = 0xff800000u;  // -inf
+    for (int p = 0; p < wk.passes() && ok; ++p) {
+        int blk, bh, n_a, n_b;
+        if (!wk.get(p, &blk, &bh, &n_a, &n_b)) continue;
+        const int n_kv = (t == 0) ? n_a : n_b;
+        const int qt = 2 * blk + t;
+        const int row = qt * kBlockQ + row_local;
+        const int qs = w % Cfg::kQStages;
+        uint8_t* stage = smem + Cfg::kOffQ + (qs * 2 + t) * Cfg::kTileBytes;  // this tile's Q buffer
+        if (n_kv == 0) {
+            // Tile entirely past the end of the sequence: only release the Q stage, and only once it
+            // has been filled, so that this warpgroup never runs ahead of the ring.
+            bool leader_ok = true;
+            if (leader) {
+                leader_ok = mbar_wait(&bars->q_full[qs], (w / Cfg::kQStages) & 1, abort_flag);
+                if (leader_ok) mbar_arrive(&bars->q_empty[qs]);
+            }
+            ok = __all_sync(0xffffffffu, leader_ok);
+            ++w;
+            continue;
         }
-        float mx0 = __uint_as_float(sr[0]), mx1 = __uint_as_float(sr[1]), mx2 = __uint_as_float(sr[2]),
-              mx3 = __uint_as_float(sr[3]);
-#pragma unroll
-        for (int i = 4; i < 128; i += 4) {
-            mx0 = fmaxf(mx0, __uint_as_float(sr[i]));
-            mx1 = fmaxf(mx1, __uint_as_float(sr[i + 1]));
-            mx2 = fmaxf(mx2, __uint_as_float(sr[i + 2]));
-            mx3 = fmaxf(mx3, __uint_as_float(sr[i + 3]));
-        }
-        const float m_tile = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+        float m_ref = -INFINITY;  // reference maximum of the raw (unscaled) scores
+        float l = 0.f;
 
-        if (j == 0) {
-            m_ref = m_tile;
-        } else {
-            const float m_new = fmaxf(m_ref, m_tile);
-            const bool grow = (m_new - m_ref) * c > kRescaleThreshold;
-            if (__any_sync(0xffffffffu, grow)) {
-                const float f = ex2_approx((m_ref - m_new) * c);  // 1 for rows whose maximum did not move
-                m_ref = m_new;
-                l *= f;
-                ok = mbar_wait(&bars->pv_done, (j - 1) & 1, abort_flag);
-                if (!ok) break;
-                tc_fence_after();
+        for (int j = 0; j < n_kv; ++j, ++cnt) {
+            ok = mbar_wait(&bars->s_full[t], cnt & 1, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            uint32_t sr[128];
+            tmem_ld_x32(t_s + 0, sr + 0);
+            tmem_ld_x32(t_s + 32, sr + 32);
+            tmem_ld_x32(t_s + 64, sr + 64);
+            tmem_ld_x32(t_s + 96, sr + 96);
+            tmem_wait_ld();
+
+            // Mask from indices only: the diagonal tile keeps key <= query; a ragged last tile keeps key < T.
+            const bool diag = kCausal && (j == qt);
+            const int keys_left = T - j * kBlockK;
+            if (diag || keys_left < kBlockK) {
+                const int lim = diag ? min(row_local, keys_left - 1) : keys_left - 1;
 #pragma unroll
-                for (int cb = 0; cb < D; cb += 32) {
-                    uint32_t o[32];
-                    tmem_ld_x32(t_o + cb, o);
-                    tmem_wait_ld();
+                for (int i = 0; i < 128; ++i)
+                    if (i > lim) sr[i] = 0xff800000u;  // -inf
+            }
+            float mx0 = __uint_as_float(sr[0]), mx1 = __uint_as_float(sr[1]), mx2 = __uint_as_float(sr[2]),
+                  mx3 = __uint_as_float(sr[3]);
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * f);
-                    tmem_st_x32(t_o + cb, o);
+            for (int i = 4; i < 128; i += 4) {
+                mx0 = fmaxf(mx0, __uint_as_float(sr[i]));
+                mx1 = fmaxf(mx1, __uint_as_float(sr[i + 1]));
+                mx2 = fmaxf(mx2, __uint_as_float(sr[i + 2]));
+                mx3 = fmaxf(mx3, __uint_as_float(sr[i + 3]));
+            }
+            const float m_tile = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+
+            if (j == 0) {
+                m_ref = m_tile;
+            } else {
+                const float m_new = fmaxf(m_ref, m_tile);
+                const bool grow = (m_new - m_ref) * c > kRescaleThreshold;
+                if (__any_sync(0xffffffffu, grow)) {
+                    const float f = ex2_approx((m_ref - m_new) * c);  // 1 for rows whose maximum did not move
+                    m_ref = m_new;
+                    l *= f;
+                    ok = mbar_wait(&bars->pv_done[t], (cnt - 1) & 1, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+#pragma unroll
+                    for (int cb = 0; cb < D; cb += 32) {
+                        uint32_t o[32];
+                        tmem_ld_x32(t_o + cb, o);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * f);
+                        tmem_st_x32(t_o + cb, o);
+                    }
                 }
             }
-        }
-        const float mc = m_ref * c;
-        float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
+            const float mc = m_ref * c;
+            float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
 #pragma unroll
-        for (int cb = 0; cb < 128; cb += 64) {
-            uint32_t pk[32];
+            for (int cb = 0; cb < 128; cb += 64) {
+                uint32_t pk[32];
 #pragma unroll
-            for (int i = 0; i < 64; i += 4) {
-                const float p0 = ex2_approx(fmaf(__uint_as_float(sr[cb + i + 0]), c, -mc));
-                const float p1 = ex2_approx(fmaf(__uint_as_float(sr[cb + i + 1]), c, -mc));
-                const float p2 = ex2_approx(fmaf(__uint_as_float(sr[cb + i + 2]), c, -mc));
-                const float p3 = ex2_approx(fmaf(__uint_as_float(sr[cb + i + 3]), c, -mc));
-                l0 += p0; l1 += p1; l2 += p2; l3 += p3;
-                pk[i / 2] = pack_bf16x2(p0, p1);
-                pk[i / 2 + 1] = pack_bf16x2(p2, p3);
+                for (int i = 0; i < 64; i += 4) {
+                    const float p0 = ex2_approx(fmaf(__uint_as_float(sr[cb + i + 0]), c, -mc));
+                    const float p1 = ex2_approx(fmaf(__uint_as_float(sr[cb + i + 1]), c, -mc));
+                    const float p2 = ex2_approx(fmaf(__uint_as_float(sr[cb + i + 2]), c, -mc));
+                    const float p3 = ex2_approx(fmaf(__uint_as_float(sr[cb + i + 3]), c, -mc));
+                    l0 += p0; l1 += p1; l2 += p2; l3 += p3;
+                    pk[i / 2] = pack_bf16x2(p0, p1);
+                    pk[i / 2 + 1] = pack_bf16x2(p2, p3);
+                }
+                tmem_st_x32(t_s + cb / 2, pk);
             }
-            tmem_st_x32(t_s + cb / 2, pk);
+            l += (l0 + l1) + (l2 + l3);
+            tmem_wait_st();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bars->p_ready[t]);
         }
-        l += (l0 + l1) + (l2 + l3);
-        tmem_wait_st();
-        tc_fence_before();
-        mbar_arrive(&bars->p_ready);
-    }
+        if (!ok) break;
 
-    if (ok) ok = mbar_wait(&bars->pv_done, (n_kv - 1) & 1, abort_flag);
-    if (!ok) return;
-    tc_fence_after();
-    const float inv_l = 1.0f / l;
-    const bool valid = row < T;
-    uint4* orow = reinterpret_cast<uint4*>(O + (static_cast<size_t>(bh) * T + row) * D);
+        // ---- end of the item: O_t / l as bf16 into this tile's Q buffer (no longer read: every
+        // Q K^T of the tile completed before its last P V), then TMA stores; LSE straight to global.
+        ok = mbar_wait(&bars->pv_done[t], (cnt - 1) & 1, abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        const float inv_l = 1.0f / l;
 #pragma unroll
-    for (int cb = 0; cb < D; cb += 32) {
-        uint32_t o[32];
-        tmem_ld_x32(t_o + cb, o);
-        tmem_wait_ld();
-        if (valid) {
+        for (int cb = 0; cb < D; cb += 32) {
+            uint32_t o[32];
+            tmem_ld_x32(t_o + cb, o);
+            tmem_wait_ld();
+            uint8_t* row_ptr = stage + (cb / 64) * kHalfTileBytes + row_local * 128;
 #pragma unroll
-            for (int i = 0; i < 32; i += 8) {
+            for (int x = 0; x < 4; ++x) {
+                const int ch = (cb % 64) / 8 + x;  // 16-byte chunk of the 128-byte swizzled row
                 uint4 v;
-                v.x = pack_bf16x2(__uint_as_float(o[i + 0]) * inv_l, __uint_as_float(o[i + 1]) * inv_l);
-                v.y = pack_bf16x2(__uint_as_float(o[i + 2]) * inv_l, __uint_as_float(o[i + 3]) * inv_l);
-                v.z = pack_bf16x2(__uint_as_float(o[i + 4]) * inv_l, __uint_as_float(o[i + 5]) * inv_l);
-                v.w = pack_bf16x2(__uint_as_float(o[i + 6]) * inv_l, __uint_as_float(o[i + 7]) * inv_l);
-                orow[(cb + i) / 8] = v;
+                v.x = pack_bf16x2(__uint_as_float(o[8 * x + 0]) * inv_l, __uint_as_float(o[8 * x + 1]) * inv_l);
+                v.y = pack_bf16x2(__uint_as_float(o[8 * x + 2]) * inv_l, __uint_as_float(o[8 * x + 3]) * inv_l);
+                v.z = pack_bf16x2(__uint_as_float(o[8 * x + 4]) * inv_l, __uint_as_float(o[8 * x + 5]) * inv_l);
+                v.w = pack_bf16x2(__uint_as_float(o[8 * x + 6]) * inv_l, __uint_as_float(o[8 * x + 7]) * inv_l);
+                *reinterpret_cast<uint4*>(row_ptr + ((ch ^ (row_local & 7)) << 4)) = v;
             }
         }
+        tc_fence_before();
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+            mbar_arrive(&bars->o_free[t]);    // O_t has been read out of TMEM
+            mbar_arrive(&bars->o_staged[t]);  // and this warp's rows are staged
+        }
+        if (row < T) LSE[static_cast<size_t>(bh) * T + row] = m_ref * scale + logf(l);
+        bool leader_ok = true;
+        if (leader) {
+            leader_ok = mbar_wait(&bars->o_staged[t], wt & 1, abort_flag);
+            if (leader_ok) {
+#pragma unroll
+                for (int h = 0; h < Cfg::kHalves; ++h)
+                    tma_store_3d(tmO, stage + h * kHalfTileBytes, h * kBoxCols, qt * kBlockQ, bh);
+                bulk_commit_group();
+                bulk_wait_group_read<0>();  // the buffer has been read and may receive the next Q tile
+                mbar_arrive(&bars->q_empty[qs]);
+            }
+        }
+        // Brings the leader back together with the rest of its warp before the next warp-wide TMEM
+        // load, and makes a failed wait of the leader a failure of the whole warp.
+        ok = __all_sync(0xffffffffu, leader_ok);
+        ++w;
+        ++wt;
     }
-    if (valid) LSE[static_cast<size_t>(bh) * T + row] = m_ref * scale + logf(l);
+    if (leader) bulk_wait_group<0>();  // O must be complete before the kernel ends
 }
 
 template <int D, bool kCausal>
-__global__ void __launch_bounds__(kFwdThreads, 2)
+__global__ void __launch_bounds__(kFwdThreads, 1)
 attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-                const __grid_constant__ CUtensorMap tmV, __nv_bfloat16* __restrict__ O, float* __restrict__ LSE,
-                int T, int BH, int n_q_tiles, float scale, int* __restrict__ dev_status) {
+                const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
+                float* __restrict__ LSE, int T, int BH, int n_blocks, float scale, int* __restrict__ dev_status) {
     using Cfg = FwdCfg<D>;
-    extern __shared__ uint8_t smem_raw[];
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     FwdBars* bars = reinterpret_cast<FwdBars*>(smem + Cfg::kOffBar);
-
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    // Heaviest query tiles (most key tiles under the causal clamp) are scheduled first.
-    const int qt = n_q_tiles - 1 - static_cast<int>(blockIdx.x) / BH;
-    const int bh = static_cast<int>(blockIdx.x) % BH;
-    const int n_kv_all = (T + kBlockK - 1) / kBlockK;
-    const int n_kv = kCausal ? min(qt + 1, n_kv_all) : n_kv_all;  // causal clamp of the key loop
+    const FwdWork wk{n_blocks * BH, static_cast<int>(gridDim.x), static_cast<int>(blockIdx.x), BH, n_blocks,
+                     (T + kBlockK - 1) / kBlockK, T, kCausal};
 
     if (threadIdx.x == 0) {
-        mbar_init(&bars->q_full, 1);
         for (int s = 0; s < 2; ++s) {
+            mbar_init(&bars->q_full[s], 1);
+            mbar_init(&bars->q_empty[s], 2);  // the store leaders of the two query tiles
             mbar_init(&bars->k_full[s], 1);
             mbar_init(&bars->k_empty[s], 1);
             mbar_init(&bars->v_full[s], 1);
             mbar_init(&bars->v_empty[s], 1);
+            mbar_init(&bars->s_full[s], 1);
+            mbar_init(&bars->p_ready[s], 4);
+            mbar_init(&bars->pv_done[s], 1);
+            mbar_init(&bars->o_free[s], 4);
+            mbar_init(&bars->o_staged[s], 4);
         }
-        mbar_init(&bars->s_full, 1);
-        mbar_init(&bars->p_ready, 128);
-        mbar_init(&bars->pv_done, 1);
         mbar_init(&bars->drain, 1);
         bars->abort_flag = 0;
         fence_mbar_init();
         tma_prefetch_desc(&tmQ);
         tma_prefetch_desc(&tmK);
         tma_prefetch_desc(&tmV);
+        tma_prefetch_desc(&tmO);
     }
     if (warp == 1) {
         tmem_alloc(&bars->tmem_base, kFwdTmemCols);
@@ -299,11 +452,12 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     const uint32_t tmem_base = bars->tmem_base;
 
     if (warp == 0) {
-        if (lane == 0) fwd_producer<D>(&tmQ, &tmK, &tmV, smem, bars, qt, bh, n_kv);
+        if (lane == 0) fwd_producer<D>(&tmQ, &tmK, &tmV, smem, bars, wk);
     } else if (warp == 1) {
-        if (lane == 0) fwd_mma<D>(smem, bars, tmem_base, n_kv);
-    } else {
-        fwd_softmax<D, kCausal>(bars, tmem_base, O, LSE, T, qt, bh, n_kv, scale, warp, lane);
+        if (lane == 0) fwd_mma<D>(smem, bars, tmem_base, wk);
+    } else if (warp >= 4) {
+        const int t = (warp - 4) >> 2;
+        fwd_softmax<D, kCausal>(smem, bars, tmem_base, &tmO, LSE, scale, wk, t, (warp - 4) & 3, lane);
     }
 
     tc_fence_before();
@@ -313,13 +467,15 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 }
 
 template <int D, bool kCausal>
-cudaError_t launch_one(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV, __nv_bfloat16* O,
-                       float* LSE, const AttnShape& s, int* dev_status, cudaStream_t stream) {
-    const int n_q_tiles = (s.T + kBlockQ - 1) / kBlockQ;
+cudaError_t launch_one(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV,
+                       const CUtensorMap& tmO, float* LSE, const AttnShape& s, int num_sms, int* dev_status,
+                       cudaStream_t stream) {
+    const int n_blocks = (s.T + kBlockRows - 1) / kBlockRows;
     const int BH = s.B * s.H;
-    const dim3 grid(static_cast<unsigned>(n_q_tiles) * BH);
+    const long long n_items = static_cast<long long>(n_blocks) * BH;
+    const dim3 grid(static_cast<unsigned>(n_items < num_sms ? n_items : num_sms));  // one persistent CTA per SM
     attn_fwd_kernel<D, kCausal><<<grid, kFwdThreads, FwdCfg<D>::kSmemBytes, stream>>>(
-        tmQ, tmK, tmV, O, LSE, s.T, BH, n_q_tiles, s.scale, dev_status);
+        tmQ, tmK, tmV, tmO, LSE, s.T, BH, n_blocks, s.scale, dev_status);
     return cudaGetLastError();
 }
 
@@ -338,14 +494,14 @@ cudaError_t configure_attn_fwd() {
 }
 
 cudaError_t launch_attn_fwd(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV,
-                            __nv_bfloat16* O, float* LSE, const AttnShape& s, int* dev_status,
+                            const CUtensorMap& tmO, float* LSE, const AttnShape& s, int num_sms, int* dev_status,
                             cudaStream_t stream) {
     if (s.D == 64) {
-        return s.causal ? launch_one<64, true>(tmQ, tmK, tmV, O, LSE, s, dev_status, stream)
-                        : launch_one<64, false>(tmQ, tmK, tmV, O, LSE, s, dev_status, stream);
+        return s.causal ? launch_one<64, true>(tmQ, tmK, tmV, tmO, LSE, s, num_sms, dev_status, stream)
+                        : launch_one<64, false>(tmQ, tmK, tmV, tmO, LSE, s, num_sms, dev_status, stream);
     }
-    return s.causal ? launch_one<128, true>(tmQ, tmK, tmV, O, LSE, s, dev_status, stream)
-                    : launch_one<128, false>(tmQ, tmK, tmV, O, LSE, s, dev_status, stream);
+    return s.causal ? launch_one<128, true>(tmQ, tmK, tmV, tmO, LSE, s, num_sms, dev_status, stream)
+                    : launch_one<128, false>(tmQ, tmK, tmV, tmO, LSE, s, num_sms, dev_status, stream);
 }
 
 }  // namespace nova

@@ -19,9 +19,10 @@ struct AttnShape {
     float scale;
 };
 
-// Forward: tensor maps are 3-D [D, T, B*H] bf16 with a [64, 128, 1] box and 128-byte swizzle.
+// Forward: tensor maps are 3-D [D, T, B*H] bf16 with a [64, 128, 1] box and 128-byte swizzle (`tmO`
+// describes the output and is used for TMA stores).  Persistent: launches at most `num_sms` CTAs.
 cudaError_t launch_attn_fwd(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV,
-                            __nv_bfloat16* O, float* LSE, const AttnShape& s, int* dev_status,
+                            const CUtensorMap& tmO, float* LSE, const AttnShape& s, int num_sms, int* dev_status,
                             cudaStream_t stream);
 cudaError_t configure_attn_fwd();
 
