@@ -196,24 +196,32 @@ __device__ __forceinline__ void bwd_mma(uint8_t* smem, BwdBars* bars, uint32_t t
     }
     const uint32_t ds_m = umma_desc_lo(smem_u32(smem + Cfg::kOffdS), kHalfTileBytes);
     uint32_t k_k = 0, v_k = 0, k_m = 0;  // per item
+    // The whole warp runs this role in uniform control flow; one elected lane issues.
+    const bool el = elect_one();
 
     auto issue_st = [&](int gq) {  // S^T = K_j Q^T for the query tile in Q stage gq & 1
         const uint32_t b = q_k[gq & 1];
+        if (el) {
 #pragma unroll
-        for (int k = 0; k < D / 16; ++k) {
-            const uint32_t off = ((k / 4) * kHalfTileBytes + (k % 4) * 32) >> 4;
-            umma_ss(t_s, umma_desc_join(k_k + off, hi), umma_desc_join(b + off, hi), kIdescT, k > 0 ? 1u : 0u);
+            for (int k = 0; k < D / 16; ++k) {
+                const uint32_t off = ((k / 4) * kHalfTileBytes + (k % 4) * 32) >> 4;
+                umma_ss(t_s, umma_desc_join(k_k + off, hi), umma_desc_join(b + off, hi), kIdescT, k > 0 ? 1u : 0u);
+            }
+            tc_commit(&bars->s_full);
         }
-        tc_commit(&bars->s_full);
+        __syncwarp();
     };
     auto issue_dpt = [&](int gq) {  // dP^T = V_j dO^T for the query tile in dO stage gq % kdOStages
         const uint32_t b = do_k[gq % Cfg::kdOStages];
+        if (el) {
 #pragma unroll
-        for (int k = 0; k < D / 16; ++k) {
-            const uint32_t off = ((k / 4) * kHalfTileBytes + (k % 4) * 32) >> 4;
-            umma_ss(t_dp, umma_desc_join(v_k + off, hi), umma_desc_join(b + off, hi), kIdescT, k > 0 ? 1u : 0u);
+            for (int k = 0; k < D / 16; ++k) {
+                const uint32_t off = ((k / 4) * kHalfTileBytes + (k % 4) * 32) >> 4;
+                umma_ss(t_dp, umma_desc_join(v_k + off, hi), umma_desc_join(b + off, hi), kIdescT, k > 0 ? 1u : 0u);
+            }
+            tc_commit(&bars->dp_full);
         }
-        tc_commit(&bars->dp_full);
+        __syncwarp();
     };
 
     bool ok = true;
@@ -253,14 +261,15 @@ __device__ __forceinline__ void bwd_mma(uint8_t* smem, BwdBars* bars, uint32_t t
                 tc_fence_after();
             }
             // dV += P^T dO_i: 16 queries (8 packed TMEM columns, 16 smem rows = 2048 bytes) per instruction.
-            {
+            if (el) {
                 const uint32_t b = do_m[g % Cfg::kdOStages];
 #pragma unroll
                 for (int k = 0; k < kBlockQ / 16; ++k)
                     umma_ts(t_dv, t_p + (k / 4) * Cfg::kPHalfStride + (k % 4) * 8, umma_desc_join(b + k * 128, hi),
                             kIdescKV, (it > 0 || k > 0) ? 1u : 0u);
+                tc_commit(&bars->do_empty[g % Cfg::kdOStages]);
             }
-            tc_commit(&bars->do_empty[g % Cfg::kdOStages]);
+            __syncwarp();
             if (!Cfg::kSeparateP && more) {  // P^T lives in the S^T columns: dV must be queued first
                 ok = mbar_wait(&bars->q_full[st ^ 1], ((g + 1) >> 1) & 1, abort_flag);
                 if (!ok) break;
@@ -270,29 +279,34 @@ __device__ __forceinline__ void bwd_mma(uint8_t* smem, BwdBars* bars, uint32_t t
             ok = mbar_wait(&bars->ds_ready, g & 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
-            {
+            if (el) {
                 const uint32_t b = q_m[st];
 #pragma unroll
                 for (int k = 0; k < kBlockQ / 16; ++k)
                     umma_ts(t_dk, t_dp + (k / 4) * 64 + (k % 4) * 8, umma_desc_join(b + k * 128, hi), kIdescKV,
                             (it > 0 || k > 0) ? 1u : 0u);
+                tc_commit(&bars->q_empty[st]);
             }
-            tc_commit(&bars->q_empty[st]);
+            __syncwarp();
             // dQ_i = dS K_j, 64 head-dim columns per accumulator half; 16 keys per instruction.
             if (!Cfg::kdQAliased) {  // the dQ warps must have read the previous tile out of the dQ columns
                 ok = mbar_wait(&bars->dq_free, (g & 1) ^ 1, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
             }
+            if (el) {
 #pragma unroll
-            for (int h = 0; h < Cfg::kHalves; ++h) {
-                const uint32_t t_dq = tmem_base + Cfg::kColdQ + h * 64;
+                for (int h = 0; h < Cfg::kHalves; ++h) {
+                    const uint32_t t_dq = tmem_base + Cfg::kColdQ + h * 64;
 #pragma unroll
-                for (int k = 0; k < kBlockK / 16; ++k)
-                    umma_ss(t_dq, umma_desc_join(ds_m + k * 128, hi),
-                            umma_desc_join(k_m + h * (kHalfTileBytes >> 4) + k * 128, hi), kIdescdQ, k > 0 ? 1u : 0u);
+                    for (int k = 0; k < kBlockK / 16; ++k)
+                        umma_ss(t_dq, umma_desc_join(ds_m + k * 128, hi),
+                                umma_desc_join(k_m + h * (kHalfTileBytes >> 4) + k * 128, hi), kIdescdQ,
+                                k > 0 ? 1u : 0u);
+                }
+                tc_commit(&bars->dq_full);
             }
-            tc_commit(&bars->dq_full);
+            __syncwarp();
             if (more) {
                 if (Cfg::kdQAliased) {  // dQ sits in the dP^T region until the dQ warps have read it
                     ok = mbar_wait(&bars->dq_free, g & 1, abort_flag);
@@ -305,13 +319,17 @@ __device__ __forceinline__ void bwd_mma(uint8_t* smem, BwdBars* bars, uint32_t t
             }
         }
         if (!ok) break;
-        tc_commit(&bars->kv_empty[ks]);  // K_j and V_j are no longer read
-        tc_commit(&bars->dkv_full);      // dV and dK of this item are complete
+        if (el) {
+            tc_commit(&bars->kv_empty[ks]);  // K_j and V_j are no longer read
+            tc_commit(&bars->dkv_full);      // dV and dK of this item are complete
+        }
+        __syncwarp();
         ++w;
     }
     if (!ok) {
         int none = 0;
-        tc_commit(&bars->drain);
+        if (el) tc_commit(&bars->drain);
+        __syncwarp();
         (void)mbar_wait(&bars->drain, 0, &none);
     }
 }
@@ -741,7 +759,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     if (warp == 0) {
         if (lane == 0) bwd_producer<D>(&tmQ, &tmK, &tmV, &tmdO, smem, bars, wl);
     } else if (warp == 1) {
-        if (lane == 0) bwd_mma<D>(smem, bars, tmem_base, wl);
+        bwd_mma<D>(smem, bars, tmem_base, wl);
     } else if (warp < 4) {
         bwd_rows(bars, reinterpret_cast<float*>(smem + Cfg::kOffRow), LSE, Delta, T, wl, (warp - 2) * 32 + lane);
     } else if (warp < 12) {

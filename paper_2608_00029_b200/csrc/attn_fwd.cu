@@ -149,6 +149,8 @@ __device__ __forceinline__ void fwd_mma(uint8_t* smem, FwdBars* bars, uint32_t t
         v_m[st] = umma_desc_lo(smem_u32(smem + Cfg::kOffV + st * Cfg::kTileBytes), kHalfTileBytes);
     }
     uint32_t q_k[2] = {0, 0};  // per item: the two query tiles
+    // The whole warp runs this role in uniform control flow; one elected lane issues.
+    const bool el = elect_one();
     bool ok = true;
     int w = 0, g = 0;
     int c[2] = {0, 0};   // key tiles processed so far per query tile (phases of its barriers)
@@ -159,12 +161,16 @@ __device__ __forceinline__ void fwd_mma(uint8_t* smem, FwdBars* bars, uint32_t t
     auto issue_qk = [&](int t, int gk) {
         const uint32_t t_s = tmem_base + Cfg::kColS + 128 * t;
         const uint32_t b = k_k[gk & 1];
+        if (el) {
 #pragma unroll
-        for (int k = 0; k < D / 16; ++k) {
-            const uint32_t off = ((k / 4) * kHalfTileBytes + (k % 4) * 32) >> 4;
-            umma_ss(t_s, umma_desc_join(q_k[t] + off, hi), umma_desc_join(b + off, hi), kIdescQK, k > 0 ? 1u : 0u);
+            for (int k = 0; k < D / 16; ++k) {
+                const uint32_t off = ((k / 4) * kHalfTileBytes + (k % 4) * 32) >> 4;
+                umma_ss(t_s, umma_desc_join(q_k[t] + off, hi), umma_desc_join(b + off, hi), kIdescQK,
+                        k > 0 ? 1u : 0u);
+            }
+            tc_commit(&bars->s_full[t]);
         }
-        tc_commit(&bars->s_full[t]);
+        __syncwarp();
     };
 
     for (int p = 0; p < wk.passes() && ok; ++p) {
@@ -183,7 +189,8 @@ __device__ __forceinline__ void fwd_mma(uint8_t* smem, FwdBars* bars, uint32_t t
         // The S columns of both tiles are free: their last P was consumed by a P V queued earlier.
         if (n_a > 0) issue_qk(0, g);
         if (n_b > 0) issue_qk(1, g);
-        tc_commit(&bars->k_empty[g & 1]);  // K tile 0 is no longer read once these have run
+        if (el) tc_commit(&bars->k_empty[g & 1]);  // K tile 0 is no longer read once these have run
+        __syncwarp();
         for (int j = 0; j < n && ok; ++j, ++g) {
             const int st = g & 1;
             bool next_k_ready = false;
@@ -205,11 +212,14 @@ __device__ __forceinline__ void fwd_mma(uint8_t* smem, FwdBars* bars, uint32_t t
                 tc_fence_after();
                 // O_t += P_t V: P from TMEM (16 keys = 8 packed columns per instruction), V is MN-major
                 // (rows = keys, 64 head-dim elements per 128-byte row, second 64-wide half at +16 KB).
+                if (el) {
 #pragma unroll
-                for (int k = 0; k < kBlockK / 16; ++k)
-                    umma_ts(t_o, t_s + k * 8, umma_desc_join(v_m[st] + k * 128, hi), kIdescPV,
-                            (j > 0 || k > 0) ? 1u : 0u);
-                tc_commit(&bars->pv_done[t]);
+                    for (int k = 0; k < kBlockK / 16; ++k)
+                        umma_ts(t_o, t_s + k * 8, umma_desc_join(v_m[st] + k * 128, hi), kIdescPV,
+                                (j > 0 || k > 0) ? 1u : 0u);
+                    tc_commit(&bars->pv_done[t]);
+                }
+                __syncwarp();
                 ++c[t];
                 if (j + 1 < n_t[t]) {  // the S_t columns are free again once this P V has run
                     if (!next_k_ready) {
@@ -222,8 +232,11 @@ __device__ __forceinline__ void fwd_mma(uint8_t* smem, FwdBars* bars, uint32_t t
                 }
             }
             if (!ok) break;
-            tc_commit(&bars->v_empty[st]);                    // V tile j is no longer read
-            if (j + 1 < n) tc_commit(&bars->k_empty[st ^ 1]);  // nor K tile j+1 (both Q K^T are queued)
+            if (el) {
+                tc_commit(&bars->v_empty[st]);                    // V tile j is no longer read
+                if (j + 1 < n) tc_commit(&bars->k_empty[st ^ 1]);  // nor K tile j+1 (both Q K^T are queued)
+            }
+            __syncwarp();
         }
         if (n_a > 0) ++wt[0];
         if (n_b > 0) ++wt[1];
@@ -232,7 +245,8 @@ __device__ __forceinline__ void fwd_mma(uint8_t* smem, FwdBars* bars, uint32_t t
     if (!ok) {
         // Drain whatever was issued before leaving so TMEM can be released safely.
         int none = 0;
-        tc_commit(&bars->drain);
+        if (el) tc_commit(&bars->drain);
+        __syncwarp();
         (void)mbar_wait(&bars->drain, 0, &none);
     }
 }
@@ -454,7 +468,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     if (warp == 0) {
         if (lane == 0) fwd_producer<D>(&tmQ, &tmK, &tmV, smem, bars, wk);
     } else if (warp == 1) {
-        if (lane == 0) fwd_mma<D>(smem, bars, tmem_base, wk);
+        fwd_mma<D>(smem, bars, tmem_base, wk);
     } else if (warp >= 4) {
         const int t = (warp - 4) >> 2;
         fwd_softmax<D, kCausal>(smem, bars, tmem_base, &tmO, LSE, scale, wk, t, (warp - 4) & 3, lane);
