@@ -16,8 +16,10 @@
 //                the final 1/sum and the LSE use the same reference maximum), and at the end of the
 //                item normalises O, stages it in the (now idle) Q tile buffer and sends it out with
 //                TMA stores.
-// TMEM columns: S_A [0,128)  S_B [128,256)  O_A [256,256+D)  O_B [256+D,256+2D); P_t is bf16 pairs
-// over the first 64 columns of S_t.
+// TMEM columns: S_A [0,128)  S_B [128,256)  O_A [256,256+D)  O_B [256+D,256+2D).  P_t (bf16 pairs,
+// 64 columns) has columns of its own at D = 64, [384,448) and [448,512): the softmax warps release
+// S_t as soon as they have loaded it, so the next Q_t K^T runs while they compute.  At D = 128 all
+// 512 columns are taken and P_t lies over the first 64 columns of S_t.
 //
 // Warp-wide .sync.aligned instructions (TMEM loads/stores) need the whole warp together: wherever
 // one lane does extra work (the store leader), the warp is rejoined with a vote before the next one.
@@ -45,12 +47,17 @@ struct FwdCfg {
     static constexpr int kSmemBytes = kOffBar + 512 + 1024;
     static constexpr int kColS = 0;      // + 128 * tile
     static constexpr int kColO = 256;    // + D * tile
+    // With D = 64 there is room for P in columns of its own, so that S_t can be overwritten by the
+    // next Q K^T as soon as the softmax warps have read it; with D = 128 P lies over S.
+    static constexpr bool kSepP = (D == 64);
+    static constexpr int kColP = kSepP ? 384 : 0;  // + 64 * tile (kSepP) / + 128 * tile
+    static constexpr int kStrideP = kSepP ? 64 : 128;
 };
 
 struct FwdBars {
     uint64_t q_full[2], q_empty[2];
     uint64_t k_full[2], k_empty[2], v_full[2], v_empty[2];
-    uint64_t s_full[2], p_ready[2], pv_done[2], o_free[2], o_staged[2];  // per query tile
+    uint64_t s_full[2], s_free[2], p_ready[2], pv_done[2], o_free[2], o_staged[2];  // per query tile
     uint64_t drain;
     uint32_t tmem_base;
     int abort_flag;
@@ -154,6 +161,7 @@ __device__ __forceinline__ void fwd_mma(uint8_t* smem, FwdBars* bars, uint32_t t
     bool ok = true;
     int w = 0, g = 0;
     int c[2] = {0, 0};   // key tiles processed so far per query tile (phases of its barriers)
+    int cq[2] = {0, 0};  // Q K^T issued so far per query tile (phases of s_free)
     int wt[2] = {0, 0};  // items in which the query tile took part so far (phases of o_free)
 
     // S_t = Q_t K^T for the key tile in stage gk & 1: both operands K-major, 16 head-dim elements
@@ -161,6 +169,12 @@ __device__ __forceinline__ void fwd_mma(uint8_t* smem, FwdBars* bars, uint32_t t
     auto issue_qk = [&](int t, int gk) {
         const uint32_t t_s = tmem_base + Cfg::kColS + 128 * t;
         const uint32_t b = k_k[gk & 1];
+        if (Cfg::kSepP && cq[t] > 0) {  // the softmax warps must have read the previous S_t
+            ok = mbar_wait(&bars->s_free[t], (cq[t] - 1) & 1, abort_flag);
+            if (!ok) return;
+            tc_fence_after();
+        }
+        ++cq[t];
         if (el) {
 #pragma unroll
             for (int k = 0; k < D / 16; ++k) {
@@ -186,18 +200,31 @@ __device__ __forceinline__ void fwd_mma(uint8_t* smem, FwdBars* bars, uint32_t t
         if (ok) ok = mbar_wait(&bars->k_full[g & 1], (g >> 1) & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
-        // The S columns of both tiles are free: their last P was consumed by a P V queued earlier.
+        // P over S: the S columns of both tiles are free, their last P was consumed by a P V queued
+        // earlier.  P apart: issue_qk waits until the previous S_t has been read.
         if (n_a > 0) issue_qk(0, g);
-        if (n_b > 0) issue_qk(1, g);
+        if (n_b > 0 && ok) issue_qk(1, g);
+        if (!ok) break;
         if (el) tc_commit(&bars->k_empty[g & 1]);  // K tile 0 is no longer read once these have run
         __syncwarp();
         for (int j = 0; j < n && ok; ++j, ++g) {
             const int st = g & 1;
             bool next_k_ready = false;
+            if (Cfg::kSepP && j + 1 < n) {
+                // Both Q K^T of the next key tile go first: S_t was released right after the softmax
+                // warps loaded it, long before their P is ready.
+                ok = mbar_wait(&bars->k_full[st ^ 1], ((g + 1) >> 1) & 1, abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+#pragma unroll
+                for (int t = 0; t < 2; ++t)
+                    if (j + 1 < n_t[t] && ok) issue_qk(t, g + 1);
+                if (!ok) break;
+            }
 #pragma unroll
             for (int t = 0; t < 2; ++t) {
                 if (j >= n_t[t]) continue;
-                const uint32_t t_s = tmem_base + Cfg::kColS + 128 * t;
+                const uint32_t t_s = tmem_base + Cfg::kColP + Cfg::kStrideP * t;
                 const uint32_t t_o = tmem_base + Cfg::kColO + D * t;
                 ok = mbar_wait(&bars->p_ready[t], c[t] & 1, abort_flag);
                 if (!ok) break;
@@ -221,7 +248,7 @@ __device__ __forceinline__ void fwd_mma(uint8_t* smem, FwdBars* bars, uint32_t t
                 }
                 __syncwarp();
                 ++c[t];
-                if (j + 1 < n_t[t]) {  // the S_t columns are free again once this P V has run
+                if (!Cfg::kSepP && j + 1 < n_t[t]) {  // the S_t columns are free again once this P V has run
                     if (!next_k_ready) {
                         ok = mbar_wait(&bars->k_full[st ^ 1], ((g + 1) >> 1) & 1, abort_flag);
                         if (!ok) break;
@@ -262,6 +289,7 @@ __device__ __forceinline__ void fwd_softmax(uint8_t* smem, FwdBars* bars, uint32
     const bool leader = (swarp == 0 && lane == 0);
     const uint32_t t_s = tmem_addr(tmem_base, lane_base, Cfg::kColS + 128 * t);
     const uint32_t t_o = tmem_addr(tmem_base, lane_base, Cfg::kColO + D * t);
+    const uint32_t t_p = tmem_addr(tmem_base, lane_base, Cfg::kColP + Cfg::kStrideP * t);
     const float c = scale * kLog2e;
     const int T = wk.T;
     bool ok = true;
@@ -300,6 +328,11 @@ __device__ __forceinline__ void fwd_softmax(uint8_t* smem, FwdBars* bars, uint32
             tmem_ld_x32(t_s + 64, sr + 64);
             tmem_ld_x32(t_s + 96, sr + 96);
             tmem_wait_ld();
+            if (Cfg::kSepP) {  // S_t may be overwritten by the next Q K^T
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&bars->s_free[t]);
+            }
 
             // Mask from indices only: the diagonal tile keeps key <= query; a ragged last tile keeps key < T.
             const bool diag = kCausal && (j == qt);
@@ -310,14 +343,16 @@ __device__ __forceinline__ void fwd_softmax(uint8_t* smem, FwdBars* bars, uint32
                 for (int i = 0; i < 128; ++i)
                     if (i > lim) sr[i] = 0xff800000u;  // -inf
             }
-            float mx0 = __uint_as_float(sr[0]), mx1 = __uint_as_float(sr[1]), mx2 = __uint_as_float(sr[2]),
-                  mx3 = __uint_as_float(sr[3]);
+            float mx0 = fmaxf(__uint_as_float(sr[0]), __uint_as_float(sr[1]));
+            float mx1 = fmaxf(__uint_as_float(sr[2]), __uint_as_float(sr[3]));
+            float mx2 = fmaxf(__uint_as_float(sr[4]), __uint_as_float(sr[5]));
+            float mx3 = fmaxf(__uint_as_float(sr[6]), __uint_as_float(sr[7]));
 #pragma unroll
-            for (int i = 4; i < 128; i += 4) {
-                mx0 = fmaxf(mx0, __uint_as_float(sr[i]));
-                mx1 = fmaxf(mx1, __uint_as_float(sr[i + 1]));
-                mx2 = fmaxf(mx2, __uint_as_float(sr[i + 2]));
-                mx3 = fmaxf(mx3, __uint_as_float(sr[i + 3]));
+            for (int i = 8; i < 128; i += 8) {
+                mx0 = fmax3(mx0, __uint_as_float(sr[i + 0]), __uint_as_float(sr[i + 1]));
+                mx1 = fmax3(mx1, __uint_as_float(sr[i + 2]), __uint_as_float(sr[i + 3]));
+                mx2 = fmax3(mx2, __uint_as_float(sr[i + 4]), __uint_as_float(sr[i + 5]));
+                mx3 = fmax3(mx3, __uint_as_float(sr[i + 6]), __uint_as_float(sr[i + 7]));
             }
             const float m_tile = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
 
@@ -333,35 +368,52 @@ __device__ __forceinline__ void fwd_softmax(uint8_t* smem, FwdBars* bars, uint32
                     ok = mbar_wait(&bars->pv_done[t], (cnt - 1) & 1, abort_flag);
                     if (!ok) break;
                     tc_fence_after();
-#pragma unroll
-                    for (int cb = 0; cb < D; cb += 32) {
-                        uint32_t o[32];
-                        tmem_ld_x32(t_o + cb, o);
+                    #pragma unroll 1
+                    for (int cb = 0; cb < D; cb += 16) {
+                        uint32_t o[16];
+                        tmem_ld_x16(t_o + cb, o);
                         tmem_wait_ld();
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * f);
-                        tmem_st_x32(t_o + cb, o);
+                        for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * f);
+                        tmem_st_x16(t_o + cb, o);
                     }
                 }
             }
-            const float mc = m_ref * c;
-            float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
+            // p = 2^(s * c - m * c): the multiply-subtract and the row sum run on packed fp32 pairs.
+            const uint64_t c2 = f32x2_pack(c, c);
+            const uint64_t nmc2 = f32x2_pack(-m_ref * c, -m_ref * c);
+            uint64_t acc0 = 0, acc1 = 0;  // two pairs of partial sums
+            if (Cfg::kSepP && j > 0) {  // the previous P_t must have been consumed (long since, as a rule)
+                ok = mbar_wait(&bars->pv_done[t], (cnt - 1) & 1, abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+            }
 #pragma unroll
             for (int cb = 0; cb < 128; cb += 64) {
                 uint32_t pk[32];
 #pragma unroll
                 for (int i = 0; i < 64; i += 4) {
-                    const float p0 = ex2_approx(fmaf(__uint_as_float(sr[cb + i + 0]), c, -mc));
-                    const float p1 = ex2_approx(fmaf(__uint_as_float(sr[cb + i + 1]), c, -mc));
-                    const float p2 = ex2_approx(fmaf(__uint_as_float(sr[cb + i + 2]), c, -mc));
-                    const float p3 = ex2_approx(fmaf(__uint_as_float(sr[cb + i + 3]), c, -mc));
-                    l0 += p0; l1 += p1; l2 += p2; l3 += p3;
+                    const uint64_t x01 = f32x2_fma(
+                        f32x2_pack(__uint_as_float(sr[cb + i + 0]), __uint_as_float(sr[cb + i + 1])), c2, nmc2);
+                    const uint64_t x23 = f32x2_fma(
+                        f32x2_pack(__uint_as_float(sr[cb + i + 2]), __uint_as_float(sr[cb + i + 3])), c2, nmc2);
+                    float x0, x1, x2, x3;
+                    f32x2_unpack(x01, x0, x1);
+                    f32x2_unpack(x23, x2, x3);
+                    const float p0 = ex2_approx(x0), p1 = ex2_approx(x1), p2 = ex2_approx(x2), p3 = ex2_approx(x3);
+                    acc0 = f32x2_add(acc0, f32x2_pack(p0, p1));
+                    acc1 = f32x2_add(acc1, f32x2_pack(p2, p3));
                     pk[i / 2] = pack_bf16x2(p0, p1);
                     pk[i / 2 + 1] = pack_bf16x2(p2, p3);
                 }
-                tmem_st_x32(t_s + cb / 2, pk);
+                tmem_st_x32(t_p + cb / 2, pk);
             }
-            l += (l0 + l1) + (l2 + l3);
+            {
+                float a0, a1, a2, a3;
+                f32x2_unpack(acc0, a0, a1);
+                f32x2_unpack(acc1, a2, a3);
+                l += (a0 + a1) + (a2 + a3);
+            }
             tmem_wait_st();
             tc_fence_before();
             __syncwarp();
@@ -443,6 +495,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             mbar_init(&bars->v_full[s], 1);
             mbar_init(&bars->v_empty[s], 1);
             mbar_init(&bars->s_full[s], 1);
+            mbar_init(&bars->s_free[s], 4);
             mbar_init(&bars->p_ready[s], 4);
             mbar_init(&bars->pv_done[s], 1);
             mbar_init(&bars->o_free[s], 4);
