@@ -403,8 +403,8 @@ __device__ __forceinline__ void fwd_softmax(uint8_t* smem, FwdBars* bars, uint32
                     const float p0 = ex2_approx(x0), p1 = ex2_approx(x1), p2 = ex2_approx(x2), p3 = ex2_approx(x3);
                     acc0 = f32x2_add(acc0, f32x2_pack(p0, p1));
                     acc1 = f32x2_add(acc1, f32x2_pack(p2, p3));
-                    pk[i / 2] = pack_bf16x2(p0, p1);
-                    pk[i / 2 + 1] = pack_bf16x2(p2, p3);
+                    pk[i / 2] = pack_bf16x2_int(p0, p1);
+                    pk[i / 2 + 1] = pack_bf16x2_int(p2, p3);
                 }
                 tmem_st_x32(t_p + cb / 2, pk);
             }
