@@ -354,7 +354,7 @@ def run_ours(args):
                        "flops_per_step": flops_step, "frac_of_burst_peak": value / world / peaks["bf16_tflops"]},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "ms_per_step": e2e_ms, "steps": e2e_steps},
-            "gpu_launches": 4 * args.steps,
+            "gpu_launches": 5 * args.steps,
             "clocks": clocks,
             "roofline": roofline,
             "cpu_baseline": cpu_baseline,

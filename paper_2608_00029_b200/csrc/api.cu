@@ -227,7 +227,7 @@ int nova_attn_bwd_steps(const void* Q, const void* K, const void* V, const void*
     float* acc = static_cast<float*>(workspace);
     cudaError_t e = cudaSuccess;
     if (steps & NOVA_ATTN_BWD_STEP_ZERO) {
-        e = cudaMemsetAsync(acc, 0, need, cs);
+        e = launch_zero(acc, need, st->num_sms, cs);
         if (e != cudaSuccess) return fail_cuda(e);
     }
     if (steps & NOVA_ATTN_BWD_STEP_MAIN) {

@@ -755,6 +755,8 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = bars->tmem_base;
+    griddep_launch_dependents();
+    griddep_wait();  // everything above overlaps the previous kernel of the stream
 
     if (warp == 0) {
         if (lane == 0) bwd_producer<D>(&tmQ, &tmK, &tmV, &tmdO, smem, bars, wl);
@@ -787,9 +789,9 @@ cudaError_t launch_one(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUt
     const int BH = s.B * s.H;
     const long long n_items = static_cast<long long>(n_tiles) * BH;
     const dim3 grid(static_cast<unsigned>(n_items < num_sms ? n_items : num_sms));  // one persistent CTA per SM
-    attn_bwd_kernel<D, kCausal><<<grid, kBwdThreads, BwdCfg<D>::kSmemBytes, stream>>>(
-        tmQ, tmK, tmV, tmdO, tmAcc, tmdK, tmdV, LSE, Delta, dq_acc, dK, dV, s.T, BH, n_tiles, s.scale, dev_status);
-    return cudaGetLastError();
+    return launch_overlapped(attn_bwd_kernel<D, kCausal>, grid, dim3(kBwdThreads), BwdCfg<D>::kSmemBytes, stream, tmQ,
+                             tmK, tmV, tmdO, tmAcc, tmdK, tmdV, LSE, Delta, dq_acc, dK, dV, s.T, BH, n_tiles, s.scale,
+                             dev_status);
 }
 
 }  // namespace

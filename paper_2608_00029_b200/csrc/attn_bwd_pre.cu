@@ -1,6 +1,7 @@
 // Memory-bound helpers of the backward pass.
 //   bwd_preprocess_kernel: Delta_i = sum_d dO[i,d] * O[i,d]   (row term of the softmax Jacobian)
 //   dq_convert_kernel:     dQ = bf16(scale * fp32 accumulator)
+//   zero_kernel:           clears the fp32 accumulator before the backward kernel adds into it
 // Both stream their inputs once with 16-byte loads; rows are split over D/8 lanes and reduced with
 // xor-shuffles.  Grids are sized in multiples of the SM count.
 #include "kernels.h"
@@ -27,6 +28,8 @@ __device__ __forceinline__ float dot8_bf16(const uint4& a, const uint4& b) {
 template <int LPR, int UNROLL>
 __global__ void __launch_bounds__(256) bwd_preprocess_kernel(const uint4* __restrict__ O, const uint4* __restrict__ dO,
                                                              float* __restrict__ Delta, long long rows) {
+    griddep_launch_dependents();
+    griddep_wait();
     const long long tid = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
     const long long nthreads = static_cast<long long>(gridDim.x) * blockDim.x;
     const long long rows_per_pass = nthreads / LPR;
@@ -58,6 +61,8 @@ __global__ void __launch_bounds__(256) bwd_preprocess_kernel(const uint4* __rest
 
 __global__ void __launch_bounds__(256) dq_convert_kernel(const float4* __restrict__ acc, uint4* __restrict__ dQ,
                                                          long long n8, float scale) {
+    griddep_launch_dependents();
+    griddep_wait();
     const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
     for (long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; i < n8; i += stride) {
         const float4 a = __ldcs(acc + 2 * i);
@@ -71,7 +76,26 @@ __global__ void __launch_bounds__(256) dq_convert_kernel(const float4* __restric
     }
 }
 
+__global__ void __launch_bounds__(256) zero_kernel(uint4* __restrict__ p, long long n16) {
+    griddep_launch_dependents();
+    griddep_wait();
+    const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
+    for (long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; i < n16; i += stride)
+        p[i] = make_uint4(0, 0, 0, 0);
+}
+
 }  // namespace
+
+cudaError_t launch_zero(void* ptr, size_t bytes, int num_sms, cudaStream_t stream) {
+    constexpr int kThreads = 256;
+    const long long n16 = static_cast<long long>(bytes / 16);
+    long long blocks = (n16 + kThreads - 1) / kThreads;
+    const long long cap = static_cast<long long>(num_sms) * 8;
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    return launch_overlapped(zero_kernel, dim3(static_cast<unsigned>(blocks)), dim3(kThreads), 0, stream,
+                             static_cast<uint4*>(ptr), n16);
+}
 
 cudaError_t launch_attn_bwd_preprocess(const __nv_bfloat16* O, const __nv_bfloat16* dO, float* Delta,
                                        long long rows, int D, int num_sms, cudaStream_t stream) {
@@ -84,11 +108,9 @@ cudaError_t launch_attn_bwd_preprocess(const __nv_bfloat16* O, const __nv_bfloat
     if (blocks < 1) blocks = 1;
     const uint4* o4 = reinterpret_cast<const uint4*>(O);
     const uint4* d4 = reinterpret_cast<const uint4*>(dO);
-    if (D == 64)
-        bwd_preprocess_kernel<8, kUnroll><<<static_cast<unsigned>(blocks), kThreads, 0, stream>>>(o4, d4, Delta, rows);
-    else
-        bwd_preprocess_kernel<16, kUnroll><<<static_cast<unsigned>(blocks), kThreads, 0, stream>>>(o4, d4, Delta, rows);
-    return cudaGetLastError();
+    const dim3 grid(static_cast<unsigned>(blocks));
+    if (D == 64) return launch_overlapped(bwd_preprocess_kernel<8, kUnroll>, grid, dim3(kThreads), 0, stream, o4, d4, Delta, rows);
+    return launch_overlapped(bwd_preprocess_kernel<16, kUnroll>, grid, dim3(kThreads), 0, stream, o4, d4, Delta, rows);
 }
 
 cudaError_t launch_dq_convert(const float* dq_acc, __nv_bfloat16* dQ, long long n, float scale, int num_sms,
@@ -99,9 +121,8 @@ cudaError_t launch_dq_convert(const float* dq_acc, __nv_bfloat16* dQ, long long 
     const long long cap = static_cast<long long>(num_sms) * 8;
     if (blocks > cap) blocks = cap;
     if (blocks < 1) blocks = 1;
-    dq_convert_kernel<<<static_cast<unsigned>(blocks), kThreads, 0, stream>>>(
-        reinterpret_cast<const float4*>(dq_acc), reinterpret_cast<uint4*>(dQ), n8, scale);
-    return cudaGetLastError();
+    return launch_overlapped(dq_convert_kernel, dim3(static_cast<unsigned>(blocks)), dim3(kThreads), 0, stream,
+                             reinterpret_cast<const float4*>(dq_acc), reinterpret_cast<uint4*>(dQ), n8, scale);
 }
 
 }  // namespace nova

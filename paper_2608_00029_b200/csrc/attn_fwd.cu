@@ -517,6 +517,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = bars->tmem_base;
+    griddep_launch_dependents();
+    griddep_wait();  // everything above overlaps the previous kernel of the stream
 
     if (warp == 0) {
         if (lane == 0) fwd_producer<D>(&tmQ, &tmK, &tmV, smem, bars, wk);
@@ -541,9 +543,8 @@ cudaError_t launch_one(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUt
     const int BH = s.B * s.H;
     const long long n_items = static_cast<long long>(n_blocks) * BH;
     const dim3 grid(static_cast<unsigned>(n_items < num_sms ? n_items : num_sms));  // one persistent CTA per SM
-    attn_fwd_kernel<D, kCausal><<<grid, kFwdThreads, FwdCfg<D>::kSmemBytes, stream>>>(
-        tmQ, tmK, tmV, tmO, LSE, s.T, BH, n_blocks, s.scale, dev_status);
-    return cudaGetLastError();
+    return launch_overlapped(attn_fwd_kernel<D, kCausal>, grid, dim3(kFwdThreads), FwdCfg<D>::kSmemBytes, stream, tmQ,
+                             tmK, tmV, tmO, LSE, s.T, BH, n_blocks, s.scale, dev_status);
 }
 
 }  // namespace

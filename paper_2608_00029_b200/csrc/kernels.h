@@ -19,6 +19,24 @@ struct AttnShape {
     float scale;
 };
 
+// Launches `kernel` allowing it to overlap the tail of the previous kernel in `stream` (programmatic
+// dependent launch); the kernel must call griddep_wait() before it touches global memory.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_overlapped(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem_bytes,
+                                     cudaStream_t stream, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem_bytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // Forward: tensor maps are 3-D [D, T, B*H] bf16 with a [64, 128, 1] box and 128-byte swizzle (`tmO`
 // describes the output and is used for TMA stores).  Persistent: launches at most `num_sms` CTAs.
 cudaError_t launch_attn_fwd(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV,
@@ -45,6 +63,9 @@ cudaError_t launch_attn_bwd(const CUtensorMap& tmQ, const CUtensorMap& tmK, cons
                             __nv_bfloat16* dK, __nv_bfloat16* dV, const AttnShape& s, int num_sms, int* dev_status,
                             cudaStream_t stream);
 cudaError_t configure_attn_bwd();
+
+// Clears `bytes` (a multiple of 16) at the 16-byte aligned `ptr`.
+cudaError_t launch_zero(void* ptr, size_t bytes, int num_sms, cudaStream_t stream);
 
 // dQ = bf16(scale * dq_acc)
 cudaError_t launch_dq_convert(const float* dq_acc, __nv_bfloat16* dQ, long long n, float scale, int num_sms,

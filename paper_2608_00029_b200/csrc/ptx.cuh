@@ -22,6 +22,18 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }
 
+// ------------------------------------------------------------------ programmatic dependent launch
+// Every kernel of the library is launched so that it may start while its predecessor in the stream
+// is still draining: its set-up (barriers, TMEM, descriptor prefetch) then overlaps the predecessor's
+// tail.  griddep_wait() blocks until the predecessor has completed and its writes are visible; nothing
+// that reads or writes global memory may come before it.  griddep_launch_dependents() lets the
+// successor be scheduled as soon as every CTA of this grid has issued it or exited.  Both are no-ops
+// in a kernel launched the ordinary way.
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void griddep_launch_dependents() {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
 // ------------------------------------------------------------------------------------------ mbarrier
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
