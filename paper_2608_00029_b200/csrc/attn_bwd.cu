@@ -199,25 +199,25 @@ __device__ __forceinline__ void bwd_mma(uint8_t* smem, BwdBars* bars, uint32_t t
     // The whole warp runs this role in uniform control flow; one elected lane issues.
     const bool el = elect_one();
 
-    auto issue_st = [&](int gq) {  // S^T = K_j Q^T for the query tile in Q stage gq & 1
+    auto issue_st = [&](int gq, uint32_t kd) {  // S^T = K Q^T: K tile `kd`, query tile in Q stage gq & 1
         const uint32_t b = q_k[gq & 1];
         if (el) {
 #pragma unroll
             for (int k = 0; k < D / 16; ++k) {
                 const uint32_t off = ((k / 4) * kHalfTileBytes + (k % 4) * 32) >> 4;
-                umma_ss(t_s, umma_desc_join(k_k + off, hi), umma_desc_join(b + off, hi), kIdescT, k > 0 ? 1u : 0u);
+                umma_ss(t_s, umma_desc_join(kd + off, hi), umma_desc_join(b + off, hi), kIdescT, k > 0 ? 1u : 0u);
             }
             tc_commit(&bars->s_full);
         }
         __syncwarp();
     };
-    auto issue_dpt = [&](int gq) {  // dP^T = V_j dO^T for the query tile in dO stage gq % kdOStages
+    auto issue_dpt = [&](int gq, uint32_t vd) {  // dP^T = V dO^T: V tile `vd`, query tile in dO stage gq % kdOStages
         const uint32_t b = do_k[gq % Cfg::kdOStages];
         if (el) {
 #pragma unroll
             for (int k = 0; k < D / 16; ++k) {
                 const uint32_t off = ((k / 4) * kHalfTileBytes + (k % 4) * 32) >> 4;
-                umma_ss(t_dp, umma_desc_join(v_k + off, hi), umma_desc_join(b + off, hi), kIdescT, k > 0 ? 1u : 0u);
+                umma_ss(t_dp, umma_desc_join(vd + off, hi), umma_desc_join(b + off, hi), kIdescT, k > 0 ? 1u : 0u);
             }
             tc_commit(&bars->dp_full);
         }
@@ -225,10 +225,19 @@ __device__ __forceinline__ void bwd_mma(uint8_t* smem, BwdBars* bars, uint32_t t
     };
 
     bool ok = true;
+    bool first_queued = false;  // S^T and dP^T of this item's first tile were queued during the previous item
     int w = 0, g = 0;
     for (int p = 0; p < wl.passes() && ok; ++p) {
         int kt, bh, i0, n_it;
         if (!wl.get(p, &kt, &bh, &i0, &n_it)) continue;
+        // With K/V double-buffered the next item's tiles arrive while this one runs, and the products
+        // of its first query tile are queued from inside this item's last iteration (below), exactly
+        // as for any other next tile: the compute warps never see the item boundary.
+        int kt_n, bh_n, i0_n, n_it_n;
+        const bool has_next = Cfg::kKVStages > 1 && p + 1 < wl.passes() && wl.get(p + 1, &kt_n, &bh_n, &i0_n, &n_it_n);
+        const int ks_n = (w + 1) % Cfg::kKVStages;
+        const uint32_t k_k_n = umma_desc_lo(smem_u32(smem + Cfg::kOffK + ks_n * Cfg::kTileBytes), 16);
+        const uint32_t v_k_n = umma_desc_lo(smem_u32(smem + Cfg::kOffV + ks_n * Cfg::kTileBytes), 16);
         const int ks = w % Cfg::kKVStages;
         k_k = umma_desc_lo(smem_u32(smem + Cfg::kOffK + ks * Cfg::kTileBytes), 16);
         k_m = umma_desc_lo(smem_u32(smem + Cfg::kOffK + ks * Cfg::kTileBytes), kHalfTileBytes);
@@ -241,19 +250,24 @@ __device__ __forceinline__ void bwd_mma(uint8_t* smem, BwdBars* bars, uint32_t t
         tc_fence_after();
         // The S^T and dP^T columns are free: the last dV / dK (and, at D=128, the dQ read-out) of the
         // previous item were queued or awaited before this point and the pipe executes in order.
-        issue_st(g);
-        issue_dpt(g);
+        if (!first_queued) {
+            issue_st(g, k_k);
+            issue_dpt(g, v_k);
+        }
+        first_queued = false;
         for (int it = 0; it < n_it && ok; ++it, ++g) {
             const int st = g & 1;
             const bool more = it + 1 < n_it;
+            const bool cross = !more && has_next && Cfg::kSeparateP && !Cfg::kdQAliased;  // next tile opens the next item
             ok = mbar_wait(&bars->p_ready, g & 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
-            if (Cfg::kSeparateP && more) {  // S^T columns are free as soon as the compute warps have read them
-                ok = mbar_wait(&bars->q_full[st ^ 1], ((g + 1) >> 1) & 1, abort_flag);
+            if (Cfg::kSeparateP && (more || cross)) {  // S^T columns are free as soon as the compute warps have read them
+                if (cross) ok = mbar_wait(&bars->kv_full[ks_n], ((w + 1) / Cfg::kKVStages) & 1, abort_flag);
+                if (ok) ok = mbar_wait(&bars->q_full[st ^ 1], ((g + 1) >> 1) & 1, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
-                issue_st(g + 1);
+                issue_st(g + 1, cross ? k_k_n : k_k);
             }
             if (it == 0 && w > 0) {  // the previous item's dV/dK have been read out of TMEM
                 ok = mbar_wait(&bars->dkv_free, (w - 1) & 1, abort_flag);
@@ -274,7 +288,7 @@ __device__ __forceinline__ void bwd_mma(uint8_t* smem, BwdBars* bars, uint32_t t
                 ok = mbar_wait(&bars->q_full[st ^ 1], ((g + 1) >> 1) & 1, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
-                issue_st(g + 1);
+                issue_st(g + 1, k_k);
             }
             ok = mbar_wait(&bars->ds_ready, g & 1, abort_flag);
             if (!ok) break;
@@ -307,7 +321,7 @@ __device__ __forceinline__ void bwd_mma(uint8_t* smem, BwdBars* bars, uint32_t t
                 tc_commit(&bars->dq_full);
             }
             __syncwarp();
-            if (more) {
+            if (more || cross) {
                 if (Cfg::kdQAliased) {  // dQ sits in the dP^T region until the dQ warps have read it
                     ok = mbar_wait(&bars->dq_free, g & 1, abort_flag);
                     if (!ok) break;
@@ -315,7 +329,8 @@ __device__ __forceinline__ void bwd_mma(uint8_t* smem, BwdBars* bars, uint32_t t
                 ok = mbar_wait(&bars->do_full[(g + 1) % Cfg::kdOStages], ((g + 1) / Cfg::kdOStages) & 1, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
-                issue_dpt(g + 1);
+                issue_dpt(g + 1, cross ? v_k_n : v_k);
+                if (cross) first_queued = true;
             }
         }
         if (!ok) break;
@@ -543,7 +558,8 @@ __device__ __forceinline__ void bwd_compute(uint8_t* smem, BwdBars* bars, uint32
 // two TMA reduce-add operations.  At the end of a work item the same warps pull dV and dK out of
 // TMEM, convert them and send them out through the same buffer with two TMA stores, so the compute
 // warps move on to the next item at once.  Nothing waits for a reduction or a store to complete
-// except the end of the kernel; the staging buffer is refilled once the copy engine has read it.
+// except the end of the kernel; before the staging buffer is refilled, the leader checks that the copy
+// engine has read it.
 __device__ __forceinline__ void bwd_dq_tma(uint8_t* smem, BwdBars* bars, uint32_t tmem_base, const CUtensorMap* tmAcc,
                                            const CUtensorMap* tmdK, const CUtensorMap* tmdV, float scale,
                                            const WorkList& wl, int qwarp, int lane) {
@@ -581,14 +597,25 @@ __device__ __forceinline__ void bwd_dq_tma(uint8_t* smem, BwdBars* bars, uint32_
                     tma_store_3d(tmdK, stage + kHalfTileBytes, 0, row, bh);
                 }
                 bulk_commit_group();
-                bulk_wait_group_read<0>();  // the staging buffer has been read and may be refilled
-                mbar_arrive(&bars->stage_free);
             }
         }
         ++u;
         // Brings the leader back together with the rest of its warp before the next warp-wide TMEM
         // load, and makes a failed wait of the leader a failure of the whole warp.
         return __all_sync(0xffffffffu, leader_ok);
+    };
+
+    // Before the staging buffer is refilled: the leader waits until the copy engine has read the
+    // previous contents.  This comes after the TMEM read-out of the new tile, so the tensor core is
+    // never held up by a copy that is still draining.
+    auto stage_reusable = [&]() -> bool {
+        if (u == 0) return true;
+        if (leader) {
+            bulk_wait_group_read<0>();
+            mbar_arrive(&bars->stage_free);
+        }
+        __syncwarp();
+        return mbar_wait(&bars->stage_free, (u - 1) & 1, abort_flag);
     };
 
     for (int p = 0; p < wl.passes() && ok; ++p) {
@@ -605,10 +632,8 @@ __device__ __forceinline__ void bwd_dq_tma(uint8_t* smem, BwdBars* bars, uint32_
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&bars->dq_free);
-            if (u >= 1) {  // the previous copy has finished reading the staging buffer
-                ok = mbar_wait(&bars->stage_free, (u - 1) & 1, abort_flag);
-                if (!ok) break;
-            }
+            ok = stage_reusable();
+            if (!ok) break;
             // fp32 [128 rows x 32 columns] per box: eight 16-byte chunks per row, 128-byte swizzle
 #pragma unroll
             for (int ch = 0; ch < 8; ++ch) {
@@ -643,10 +668,8 @@ __device__ __forceinline__ void bwd_dq_tma(uint8_t* smem, BwdBars* bars, uint32_
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(&bars->dkv_free);
-        if (u >= 1) {
-            ok = mbar_wait(&bars->stage_free, (u - 1) & 1, abort_flag);
-            if (!ok) break;
-        }
+        ok = stage_reusable();
+        if (!ok) break;
 #pragma unroll
         for (int ch = 0; ch < 8; ++ch) {
             *reinterpret_cast<uint4*>(row0 + ((ch ^ sw) << 4)) =
