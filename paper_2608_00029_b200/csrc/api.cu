@@ -240,7 +240,7 @@ int nova_attn_bwd_steps(const void* Q, const void* K, const void* V, const void*
         if (int rc = get_tensor_map(dK, D, T, BH, &tmdK)) return rc;
         if (int rc = get_tensor_map(dV, D, T, BH, &tmdV)) return rc;
         const AttnShape s{B, H, T, D, causal != 0, scale};
-        e = launch_attn_bwd(tmQ, tmK, tmV, tmdO, tmAcc, tmdK, tmdV, LSE, Delta, acc, static_cast<__nv_bfloat16*>(dK),
+        e = launch_attn_bwd(tmQ, tmK, tmV, tmdO, tmAcc, tmdK, tmdV, LSE, Delta, static_cast<__nv_bfloat16*>(dK),
                             static_cast<__nv_bfloat16*>(dV), s, st->num_sms, st->dev_status, cs);
         if (e != cudaSuccess) return fail_cuda(e);
     }

@@ -26,8 +26,8 @@
 //   warps 4-11   compute: thread = (key row, 64-query half); P phase then dS phase per tile
 //                (at D=128 they also write dV and dK at the end of an item)
 //   warps 12-15  dQ: one thread per row moves the partial dQ tile from TMEM into the fp32 accumulator
-//                (TMA reduce-add through a swizzled staging buffer at D=64, red.global.add.v4.f32 at
-//                D=128; a separate kernel scales and rounds it once); at D=64 they also send dV and dK
+//                with TMA reduce-add operations through a swizzled staging buffer (a separate kernel
+//                scales and rounds it once); at D=64 they also send dV and dK
 //                of a finished item out through the same buffer with TMA stores
 //
 // TMEM columns (D=64): S^T [0,128)  dP^T/dS^T [128,256)  dV [256,320)  dK [320,384)  dQ [384,448)
@@ -61,13 +61,19 @@ struct BwdCfg {
     static constexpr int kOffdO = kOffQ + 2 * kTileBytes;             // kdOStages stages
     static constexpr int kOffdS = kOffdO + kdOStages * kTileBytes;    // [2 query halves][128 keys][64 queries] bf16
     static constexpr int kOffRow = kOffdS + 2 * kHalfTileBytes;       // 2 x (LSE*log2e[128], Delta[128]) fp32
-    // Staging buffer of the dQ warps (D=64 only): two boxes of [128 rows x 128 bytes], 128-byte
-    // swizzled like every other tile (fp32 [128 x 32] each for dQ, bf16 [128 x 64] each for dV, dK).
+    // Staging buffer of the dQ warps: two boxes of [128 rows x 128 bytes], 128-byte swizzled like every
+    // other tile (fp32 [128 x 32] each for dQ; at D=64 also bf16 [128 x 64] each for dV and dK, which the
+    // dQ warps then send out too: kBulkdQ).
     static constexpr bool kBulkdQ = (D == 64);
     static constexpr int kStageBytes = 2 * kHalfTileBytes;
     static constexpr int kOffStage = kOffRow + 2 * 2 * 128 * 4;
-    static constexpr int kOffBar = kOffStage + (kBulkdQ ? kStageBytes : 0);
-    static constexpr int kSmemBytes = kOffBar + 512 + 1024;
+    static constexpr int kOffBar = kOffStage + kStageBytes;
+    // At D=128 the tiles fill the 227 KB a CTA can have to within 512 bytes, so there is no room for
+    // the padding that would let the kernel align its window itself: the kernel checks that the window
+    // starts on a 1024-byte boundary (it does on sm_100) and gives up cleanly if not.
+    static constexpr int kAlignPad = (D == 64) ? 1024 : 0;
+    static constexpr int kSmemBytes = kOffBar + 512 + kAlignPad;
+    static_assert(kSmemBytes <= 232448, "exceeds the shared memory of one CTA");
     static constexpr int kColS = 0;
     static constexpr int kColdP = 128;
     static constexpr int kColdV = 256;
@@ -685,41 +691,83 @@ __device__ __forceinline__ void bwd_dq_tma(uint8_t* smem, BwdBars* bars, uint32_
     if (leader) bulk_wait_group<0>();
 }
 
-// dQ warps at D=128: one thread per query row adds its partial row with red.global.add.v4.f32.
-__device__ __forceinline__ void bwd_dq_red(BwdBars* bars, uint32_t tmem_base, float* __restrict__ dq_acc, int T,
-                                           const WorkList& wl, int qwarp, int lane) {
+// dQ warps at D=128.  One thread per query row; the partial dQ tile is 128 fp32 columns, i.e. four
+// boxes of the accumulator's tensor map.  They leave TMEM two at a time (64 registers), go through the
+// two halves of the staging buffer and out with one TMA reduce-add each; the dQ columns are released
+// as soon as the second pair has been loaded, and a half of the buffer is refilled once the copy
+// engine has read the box before last.
+__device__ __forceinline__ void bwd_dq_tma_wide(uint8_t* smem, BwdBars* bars, uint32_t tmem_base,
+                                                const CUtensorMap* tmAcc, const WorkList& wl, int qwarp, int lane) {
     constexpr int D = 128;
     using Cfg = BwdCfg<D>;
     volatile int* abort_flag = &bars->abort_flag;
     const uint32_t lane_base = 32u * (qwarp & 3);
-    const int r = lane_base + lane;
-    int g = 0;
-    for (int p = 0; p < wl.passes(); ++p) {
+    const int r = lane_base + lane;  // local query row
+    const bool leader = (qwarp == 0 && lane == 0);
+    const uint32_t t_dq = tmem_addr(tmem_base, lane_base, Cfg::kColdQ);
+    uint8_t* stage = smem + Cfg::kOffStage;
+    const int sw = r & 7;
+    bool ok = true;
+    int g = 0, u = 0;  // query tiles, boxes sent so far
+
+    // Sends 32 accumulator columns (one box) of this thread's row through half (u & 1) of the buffer.
+    auto send_box = [&](const uint32_t* a, int col, int row, int bh) -> bool {
+        if (u >= 2) {  // the box before last used this half: the copy engine must have read it
+            if (leader) {
+                bulk_wait_group_read<1>();
+                mbar_arrive(&bars->stage_free);
+            }
+            __syncwarp();
+            if (!mbar_wait(&bars->stage_free, (u - 2) & 1, abort_flag)) return false;
+        }
+        uint8_t* box = stage + (u & 1) * kHalfTileBytes;
+        uint8_t* row_ptr = box + r * 128;
+#pragma unroll
+        for (int ch = 0; ch < 8; ++ch)
+            *reinterpret_cast<uint4*>(row_ptr + ((ch ^ sw) << 4)) =
+                make_uint4(a[ch * 4], a[ch * 4 + 1], a[ch * 4 + 2], a[ch * 4 + 3]);
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&bars->stage_full);
+        bool leader_ok = true;
+        if (leader) {
+            leader_ok = mbar_wait(&bars->stage_full, u & 1, abort_flag);
+            if (leader_ok) {
+                tma_reduce_add_3d(tmAcc, box, col, row, bh);
+                bulk_commit_group();
+            }
+        }
+        ++u;
+        return __all_sync(0xffffffffu, leader_ok);
+    };
+
+    for (int p = 0; p < wl.passes() && ok; ++p) {
         int kt, bh, i0, n_it;
         if (!wl.get(p, &kt, &bh, &i0, &n_it)) continue;
-        const size_t row_base = static_cast<size_t>(bh) * T;
-        for (int it = 0; it < n_it; ++it, ++g) {
-            if (!mbar_wait(&bars->dq_full, g & 1, abort_flag)) return;
+        for (int it = 0; it < n_it && ok; ++it, ++g) {
+            ok = mbar_wait(&bars->dq_full, g & 1, abort_flag);
+            if (!ok) break;
             tc_fence_after();
-            const int q = (i0 + it) * kBlockQ + r;
-            float* dst = dq_acc + (row_base + q) * D;
+            const int row = (i0 + it) * kBlockQ;
 #pragma unroll
-            for (int cb = 0; cb < D; cb += 32) {
-                uint32_t a[32];
-                tmem_ld_x32(tmem_addr(tmem_base, lane_base, Cfg::kColdQ + cb), a);
+            for (int half = 0; half < 2 && ok; ++half) {
+                uint32_t a[64];
+                tmem_ld_x32(t_dq + 64 * half, a);
+                tmem_ld_x32(t_dq + 64 * half + 32, a + 32);
                 tmem_wait_ld();
-                if (q < T) {
-#pragma unroll
-                    for (int x = 0; x < 32; x += 4)
-                        red_add_v4_f32(dst + cb + x, __uint_as_float(a[x]), __uint_as_float(a[x + 1]),
-                                       __uint_as_float(a[x + 2]), __uint_as_float(a[x + 3]));
+                if (half == 1) {  // the whole tile has left TMEM
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&bars->dq_free);
                 }
+                ok = send_box(a, 64 * half, row, bh);
+                if (ok) ok = send_box(a + 32, 64 * half + 32, row, bh);
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&bars->dq_free);
         }
     }
+    // Also when giving up: nothing of this thread may stay in flight, and the accumulator must be
+    // complete before the kernel ends.
+    if (leader) bulk_wait_group<0>();
 }
 
 template <int D, bool kCausal>
@@ -728,12 +776,16 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmdO,
                 const __grid_constant__ CUtensorMap tmAcc, const __grid_constant__ CUtensorMap tmdK,
                 const __grid_constant__ CUtensorMap tmdV, const float* __restrict__ LSE,
-                const float* __restrict__ Delta, float* __restrict__ dq_acc, __nv_bfloat16* __restrict__ dK,
+                const float* __restrict__ Delta, __nv_bfloat16* __restrict__ dK,
                 __nv_bfloat16* __restrict__ dV, int T, int BH, int n_tiles, float scale,
                 int* __restrict__ dev_status) {
     using Cfg = BwdCfg<D>;
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    if (Cfg::kAlignPad == 0 && smem != smem_raw) {  // no room to realign: give up before anything is set up
+        if (threadIdx.x == 0) atomicExch(dev_status, kDevTimeout);
+        return;
+    }
     BwdBars* bars = reinterpret_cast<BwdBars*>(smem + Cfg::kOffBar);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const WorkList wl{n_tiles * BH, static_cast<int>(gridDim.x), static_cast<int>(blockIdx.x), BH, n_tiles, kCausal};
@@ -793,7 +845,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         if constexpr (Cfg::kBulkdQ)
             bwd_dq_tma(smem, bars, tmem_base, &tmAcc, &tmdK, &tmdV, scale, wl, warp - 12, lane);
         else
-            bwd_dq_red(bars, tmem_base, dq_acc, T, wl, warp - 12, lane);
+            bwd_dq_tma_wide(smem, bars, tmem_base, &tmAcc, wl, warp - 12, lane);
     }
 
     tc_fence_before();
@@ -805,7 +857,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 template <int D, bool kCausal>
 cudaError_t launch_one(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV,
                        const CUtensorMap& tmdO, const CUtensorMap& tmAcc, const CUtensorMap& tmdK,
-                       const CUtensorMap& tmdV, const float* LSE, const float* Delta, float* dq_acc,
+                       const CUtensorMap& tmdV, const float* LSE, const float* Delta,
                        __nv_bfloat16* dK, __nv_bfloat16* dV, const AttnShape& s, int num_sms, int* dev_status,
                        cudaStream_t stream) {
     const int n_tiles = (s.T + kBlockK - 1) / kBlockK;
@@ -813,7 +865,7 @@ cudaError_t launch_one(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUt
     const long long n_items = static_cast<long long>(n_tiles) * BH;
     const dim3 grid(static_cast<unsigned>(n_items < num_sms ? n_items : num_sms));  // one persistent CTA per SM
     return launch_overlapped(attn_bwd_kernel<D, kCausal>, grid, dim3(kBwdThreads), BwdCfg<D>::kSmemBytes, stream, tmQ,
-                             tmK, tmV, tmdO, tmAcc, tmdK, tmdV, LSE, Delta, dq_acc, dK, dV, s.T, BH, n_tiles, s.scale,
+                             tmK, tmV, tmdO, tmAcc, tmdK, tmdV, LSE, Delta, dK, dV, s.T, BH, n_tiles, s.scale,
                              dev_status);
 }
 
@@ -833,15 +885,15 @@ cudaError_t configure_attn_bwd() {
 
 cudaError_t launch_attn_bwd(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV,
                             const CUtensorMap& tmdO, const CUtensorMap& tmAcc, const CUtensorMap& tmdK,
-                            const CUtensorMap& tmdV, const float* LSE, const float* Delta, float* dq_acc,
+                            const CUtensorMap& tmdV, const float* LSE, const float* Delta,
                             __nv_bfloat16* dK, __nv_bfloat16* dV, const AttnShape& s, int num_sms, int* dev_status,
                             cudaStream_t stream) {
     if (s.D == 64) {
-        return s.causal ? launch_one<64, true>(tmQ, tmK, tmV, tmdO, tmAcc, tmdK, tmdV, LSE, Delta, dq_acc, dK, dV, s, num_sms, dev_status, stream)
-                        : launch_one<64, false>(tmQ, tmK, tmV, tmdO, tmAcc, tmdK, tmdV, LSE, Delta, dq_acc, dK, dV, s, num_sms, dev_status, stream);
+        return s.causal ? launch_one<64, true>(tmQ, tmK, tmV, tmdO, tmAcc, tmdK, tmdV, LSE, Delta, dK, dV, s, num_sms, dev_status, stream)
+                        : launch_one<64, false>(tmQ, tmK, tmV, tmdO, tmAcc, tmdK, tmdV, LSE, Delta, dK, dV, s, num_sms, dev_status, stream);
     }
-    return s.causal ? launch_one<128, true>(tmQ, tmK, tmV, tmdO, tmAcc, tmdK, tmdV, LSE, Delta, dq_acc, dK, dV, s, num_sms, dev_status, stream)
-                    : launch_one<128, false>(tmQ, tmK, tmV, tmdO, tmAcc, tmdK, tmdV, LSE, Delta, dq_acc, dK, dV, s, num_sms, dev_status, stream);
+    return s.causal ? launch_one<128, true>(tmQ, tmK, tmV, tmdO, tmAcc, tmdK, tmdV, LSE, Delta, dK, dV, s, num_sms, dev_status, stream)
+                    : launch_one<128, false>(tmQ, tmK, tmV, tmdO, tmAcc, tmdK, tmdV, LSE, Delta, dK, dV, s, num_sms, dev_status, stream);
 }
 
 }  // namespace nova

@@ -53,13 +53,13 @@ cudaError_t launch_attn_delta(const CUtensorMap& tmQ, const CUtensorMap& tmK, co
                               int* dev_status, cudaStream_t stream);
 cudaError_t configure_attn_delta();
 
-// Backward main kernel: adds unscaled dQ partial tiles into `dq_acc` (fp32 [B,H,T,D], zero on entry; also
-// described by `tmAcc`: fp32 [D, T, B*H], box [32, 128, 1], 128-byte swizzle) and writes dK and dV
+// Backward main kernel: adds unscaled dQ partial tiles into the fp32 accumulator [B,H,T,D] (zero on
+// entry) described by `tmAcc` (fp32 [D, T, B*H], box [32, 128, 1], 128-byte swizzle) and writes dK and dV
 // (`tmdK`, `tmdV`: the usual bf16 maps of the outputs, used for TMA stores at D=64).
 // Persistent: launches at most `num_sms` CTAs.
 cudaError_t launch_attn_bwd(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV,
                             const CUtensorMap& tmdO, const CUtensorMap& tmAcc, const CUtensorMap& tmdK,
-                            const CUtensorMap& tmdV, const float* LSE, const float* Delta, float* dq_acc,
+                            const CUtensorMap& tmdV, const float* LSE, const float* Delta,
                             __nv_bfloat16* dK, __nv_bfloat16* dV, const AttnShape& s, int num_sms, int* dev_status,
                             cudaStream_t stream);
 cudaError_t configure_attn_bwd();

@@ -60,19 +60,6 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     return ok != 0;
 }
 
-// Non-blocking test of the phase with the given parity (never suspends the thread).
-__device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-
 // Same test, but the hardware may keep the thread suspended for up to `hint_ns` while the phase is
 // incomplete (it resumes at once when the phase completes).  A suspended thread issues nothing, so
 // waiting warps do not take issue slots from the warps that share their scheduler.
@@ -284,11 +271,6 @@ __device__ __forceinline__ float ex2_approx(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
-__device__ __forceinline__ float lg2_approx(float x) {
-    float y;
-    asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
 // Packed pairs of fp32 in one 64-bit register: sm_100 executes fma/add on both halves in one
 // instruction, which halves the issue slots of the softmax arithmetic.
 __device__ __forceinline__ uint64_t f32x2_pack(float lo, float hi) {
@@ -309,11 +291,6 @@ __device__ __forceinline__ uint64_t f32x2_add(uint64_t a, uint64_t b) {
     asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
     return r;
 }
-__device__ __forceinline__ uint64_t f32x2_mul(uint64_t a, uint64_t b) {
-    uint64_t r;
-    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
-    return r;
-}
 // max of three in one instruction
 __device__ __forceinline__ float fmax3(float a, float b, float c) {
     float r;
@@ -331,17 +308,6 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 // (a tie is one fp32 value in 65536, so the difference from round-to-nearest-even does not bias sums).
 __device__ __forceinline__ uint32_t pack_bf16x2_int(float lo, float hi) {
     return __byte_perm(__float_as_uint(lo) + 0x8000u, __float_as_uint(hi) + 0x8000u, 0x7632);
-}
-__device__ __forceinline__ void red_add_v4_f32(float* addr, float a, float b, float c, float d) {
-    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(a), "f"(b), "f"(c), "f"(d)
-                 : "memory");
-}
-// Bulk asynchronous reduction shared -> global: global[i] += smem[i] for `bytes`/4 floats, performed
-// by the copy engine at L2.  Both addresses 16-byte aligned, `bytes` a multiple of 16.
-__device__ __forceinline__ void bulk_reduce_add_f32(float* gdst, const void* smem_src, uint32_t bytes) {
-    asm volatile("cp.reduce.async.bulk.global.shared::cta.bulk_group.add.f32 [%0], [%1], %2;" ::"l"(gdst),
-                 "r"(smem_u32(smem_src)), "r"(bytes)
-                 : "memory");
 }
 __device__ __forceinline__ void bulk_commit_group() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 // At most N of this thread's bulk groups still pending (.read: only their shared-memory reads).
