@@ -291,11 +291,15 @@ def run_ours(args):
         "preprocess_gbs": (4.0 * cfg.B * cfg.H * cfg.T * cfg.D + 4.0 * cfg.B * cfg.H * cfg.T)
         / (kernel_ms["bwd_preprocess"] * 1e-3) / 1e9,
     }
-    traffic_path = os.path.join(ROOT, "profiles", "traffic.json")
-    if os.path.exists(traffic_path):
+    # DRAM bytes of one launch of the dominant kernel, from the committed ncu summary of this workload
+    # (a "traffic_bytes_per_launch: N" line); absent or another workload -> null.
+    traffic_path = os.path.join(ROOT, "profiles", f"attn_bwd_kernel_{base.name}.md")
+    if os.path.exists(traffic_path) and cfg.B == base.B:
         try:
             with open(traffic_path) as f:
-                roofline["traffic"] = json.load(f).get("attn_bwd_kernel_bytes_per_launch")
+                for line in f:
+                    if line.startswith("traffic_bytes_per_launch:"):
+                        roofline["traffic"] = int(line.split(":")[1])
         except Exception:
             pass
 

@@ -22,9 +22,13 @@
  *     memory.
  *   - Return value: NOVA_ATTN_OK (0) or a negative nova_attn_status.  Arguments are validated on the
  *     host before anything is launched; a failed call has launched nothing.
- *   - Every wait inside the kernels is bounded.  If one expires (which indicates a bug or a broken
- *     device, never a property of the input) the kernel records NOVA_ATTN_ERR_TIMEOUT in a device
- *     status word, releases what it holds and returns; nova_attn_poll_device_status() reads the word.
+ *   - Every wait inside the kernels is bounded.  If one expires, or a kernel finds at start-up that it
+ *     cannot run as built (both indicate a bug or a broken device, never a property of the input), the
+ *     kernel records NOVA_ATTN_ERR_TIMEOUT in a device status word, releases what it holds and returns;
+ *     nova_attn_poll_device_status() reads the word.
+ *   - Kernels are launched so that each may begin its set-up while the previous kernel in `stream` is
+ *     still draining (programmatic dependent launch); each waits for its predecessor before it reads or
+ *     writes global memory, so stream order is what the caller observes.
  */
 #ifndef NOVA_ATTN_H_
 #define NOVA_ATTN_H_
@@ -103,9 +107,9 @@ size_t nova_attn_bwd_workspace_bytes(int B, int H, int T, int D);
  *   dQ, dK, dV  : out, bf16 [B,H,T,D]; gradient of sum(O * dO) with respect to Q, K, V
  *   workspace   : device scratch of at least nova_attn_bwd_workspace_bytes(B,H,T,D) bytes, 16-byte
  *                 aligned; zeroed by the call itself on `stream`; contents afterwards unspecified.
- * dQ is accumulated in fp32 across key tiles with floating-point atomics, so its low-order bits may
- * differ from run to run; dK and dV are deterministic.  A final pass scales the accumulator, rounds it
- * once to bf16 and writes dQ.
+ * dQ is accumulated in fp32 across key tiles with floating-point reduce-adds whose order is not fixed,
+ * so its low-order bits may differ from run to run; dK and dV are deterministic.  A final pass scales
+ * the accumulator, rounds it once to bf16 and writes dQ.
  */
 int nova_attn_bwd(const void* Q, const void* K, const void* V, const void* O, const void* dO,
                   const float* LSE, const float* Delta, void* dQ, void* dK, void* dV,
