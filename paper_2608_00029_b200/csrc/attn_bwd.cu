@@ -22,7 +22,7 @@
 //   warp 1       UMMA issuer, software-pipelined: S^T of the next query tile is issued as soon as the
 //                compute warps have read the current one; dK, dQ and the next dP^T run while they
 //                work on the next P
-//   warps 2-3    row loader: LSE*log2e and Delta of the query tile into shared memory
+//   warps 2-3    row loader: -LSE*log2e and -Delta of the query tile into shared memory
 //   warps 4-11   compute: thread = (key row, 64-query half); P phase then dS phase per tile
 //                (at D=128 they also write dV and dK at the end of an item)
 //   warps 12-15  dQ: one thread per row moves the partial dQ tile from TMEM into the fp32 accumulator
@@ -60,7 +60,7 @@ struct BwdCfg {
     static constexpr int kOffQ = 2 * kKVStages * kTileBytes;          // 2 stages
     static constexpr int kOffdO = kOffQ + 2 * kTileBytes;             // kdOStages stages
     static constexpr int kOffdS = kOffdO + kdOStages * kTileBytes;    // [2 query halves][128 keys][64 queries] bf16
-    static constexpr int kOffRow = kOffdS + 2 * kHalfTileBytes;       // 2 x (LSE*log2e[128], Delta[128]) fp32
+    static constexpr int kOffRow = kOffdS + 2 * kHalfTileBytes;       // 2 x (-LSE*log2e[128], -Delta[128]) fp32
     // Staging buffer of the dQ warps: two boxes of [128 rows x 128 bytes], 128-byte swizzled like every
     // other tile (fp32 [128 x 32] each for dQ; at D=64 also bf16 [128 x 64] each for dV and dK, which the
     // dQ warps then send out too: kBulkdQ).
@@ -355,7 +355,8 @@ __device__ __forceinline__ void bwd_mma(uint8_t* smem, BwdBars* bars, uint32_t t
     }
 }
 
-// Row loader: LSE*log2e and Delta of each query tile into the double-buffered row arrays.
+// Row loader: -LSE*log2e and -Delta of each query tile into the double-buffered row arrays (negated,
+// so that the compute warps fold them in with a packed fma / add).
 __device__ __forceinline__ void bwd_rows(BwdBars* bars, float* row_buf, const float* __restrict__ LSE,
                                          const float* __restrict__ Delta, int T, const WorkList& wl, int tid64) {
     volatile int* abort_flag = &bars->abort_flag;
@@ -374,8 +375,8 @@ __device__ __forceinline__ void bwd_rows(BwdBars* bars, float* row_buf, const fl
                 const int rl = tid64 + 64 * x;
                 const int q = (i0 + it) * kBlockQ + rl;
                 // Rows past the end of the sequence get LSE = +inf so that their P is exactly 0.
-                s_lse[rl] = (q < T) ? LSE[row_base + q] * kLog2e : INFINITY;
-                s_dl[rl] = (q < T) ? Delta[row_base + q] : 0.f;
+                s_lse[rl] = (q < T) ? -LSE[row_base + q] * kLog2e : -INFINITY;
+                s_dl[rl] = (q < T) ? -Delta[row_base + q] : 0.f;
             }
             __syncwarp();
             if ((tid64 & 31) == 0) mbar_arrive(&bars->row_full[b]);
@@ -383,7 +384,8 @@ __device__ __forceinline__ void bwd_rows(BwdBars* bars, float* row_buf, const fl
     }
 }
 
-// P phase for this thread's 64 queries: p = exp2(s*c - lse*log2e), packed to bf16 pairs.
+// P phase for this thread's 64 queries: p = exp2(s*c - lse*log2e), packed to bf16 pairs.  `s_lse4`
+// holds -lse*log2e; the multiply-add runs on packed fp32 pairs.
 // kMasked: the tile is the diagonal one and/or holds keys past the end of the sequence.
 template <bool kMasked>
 __device__ __forceinline__ void bwd_p_phase(const uint32_t (&sv)[64], const float4* s_lse4, float c, uint32_t (&pk)[32],
@@ -391,10 +393,13 @@ __device__ __forceinline__ void bwd_p_phase(const uint32_t (&sv)[64], const floa
 #pragma unroll
     for (int g = 0; g < 16; ++g) {
         const float4 l4 = s_lse4[g];
-        float p0 = ex2_approx(fmaf(__uint_as_float(sv[4 * g + 0]), c, -l4.x));
-        float p1 = ex2_approx(fmaf(__uint_as_float(sv[4 * g + 1]), c, -l4.y));
-        float p2 = ex2_approx(fmaf(__uint_as_float(sv[4 * g + 2]), c, -l4.z));
-        float p3 = ex2_approx(fmaf(__uint_as_float(sv[4 * g + 3]), c, -l4.w));
+        const uint64_t c2 = f32x2_pack(c, c);
+        float x0, x1, x2, x3;
+        f32x2_unpack(f32x2_fma(f32x2_pack(__uint_as_float(sv[4 * g + 0]), __uint_as_float(sv[4 * g + 1])), c2,
+                               f32x2_pack(l4.x, l4.y)), x0, x1);
+        f32x2_unpack(f32x2_fma(f32x2_pack(__uint_as_float(sv[4 * g + 2]), __uint_as_float(sv[4 * g + 3])), c2,
+                               f32x2_pack(l4.z, l4.w)), x2, x3);
+        float p0 = ex2_approx(x0), p1 = ex2_approx(x1), p2 = ex2_approx(x2), p3 = ex2_approx(x3);
         if (kMasked) {
             // keep (query q, key r) iff the key exists and, on the diagonal tile, key <= query
             const int q0 = q_base + 4 * g;
@@ -508,10 +513,14 @@ __device__ __forceinline__ void bwd_compute(uint8_t* smem, BwdBars* bars, uint32
                     const uint32_t pa = pk[2 * x], pb = pk[2 * x + 1];
                     const float p0 = __uint_as_float(pa << 16), p1 = __uint_as_float(pa & 0xffff0000u);
                     const float p2 = __uint_as_float(pb << 16), p3 = __uint_as_float(pb & 0xffff0000u);
-                    const float d0 = p0 * (__uint_as_float(dv[4 * x + 0]) - d4.x);
-                    const float d1 = p1 * (__uint_as_float(dv[4 * x + 1]) - d4.y);
-                    const float d2 = p2 * (__uint_as_float(dv[4 * x + 2]) - d4.z);
-                    const float d3 = p3 * (__uint_as_float(dv[4 * x + 3]) - d4.w);
+                    // d4 holds -delta: ds = p * (dp + (-delta)) on packed fp32 pairs
+                    float d0, d1, d2, d3;
+                    f32x2_unpack(f32x2_mul(f32x2_pack(p0, p1),
+                                           f32x2_add(f32x2_pack(__uint_as_float(dv[4 * x + 0]), __uint_as_float(dv[4 * x + 1])),
+                                                     f32x2_pack(d4.x, d4.y))), d0, d1);
+                    f32x2_unpack(f32x2_mul(f32x2_pack(p2, p3),
+                                           f32x2_add(f32x2_pack(__uint_as_float(dv[4 * x + 2]), __uint_as_float(dv[4 * x + 3])),
+                                                     f32x2_pack(d4.z, d4.w))), d2, d3);
                     dd[2 * x + 0] = pack_bf16x2(d0, d1);
                     dd[2 * x + 1] = pack_bf16x2(d2, d3);
                 }
