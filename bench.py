@@ -310,23 +310,46 @@ def run_ours(args):
     h2d = sum(x.numel() * x.element_size() for x in host_in[0])
     d2h = sum(x.numel() * x.element_size() for x in host_out[0])
 
+    # Three streams, as a caller that feeds the library from the host would run it: the copies of step
+    # i+1's inputs and of step i-1's results overlap step i's kernels (PCIe is full duplex).  Every step
+    # still moves all of its inputs in and all of its results out inside the timed region.
+    s_in, s_out = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+    set_free = [None] * n_sets  # event: the results of the last step that used the set have left the device
+
     def e2e_step(i):
-        s = sets[i % n_sets]
+        k = i % n_sets
+        s = sets[k]
         hi, ho = host_in[i % 2], host_out[i % 2]
-        for dst, src in zip((s.q, s.k, s.v, s.do), hi):
-            dst.copy_(src, non_blocking=True)
+        with torch.cuda.stream(s_in):
+            if set_free[k] is not None:
+                s_in.wait_event(set_free[k])
+            for dst, src in zip((s.q, s.k, s.v, s.do), hi):
+                dst.copy_(src, non_blocking=True)
+            in_ready = s_in.record_event()
+        stream.wait_event(in_ready)
         step(na, cfg, s)
-        for dst, src in zip(ho, (s.o, s.dq, s.dk, s.dv)):
-            dst.copy_(src, non_blocking=True)
+        done = stream.record_event()
+        with torch.cuda.stream(s_out):
+            s_out.wait_event(done)
+            for dst, src in zip(ho, (s.o, s.dq, s.dk, s.dv)):
+                dst.copy_(src, non_blocking=True)
+            set_free[k] = s_out.record_event()
+
+    def e2e_join():  # the launching stream waits for the copies still in flight
+        for e in set_free:
+            if e is not None:
+                stream.wait_event(e)
 
     e2e_steps = max(3, min(args.steps, 50))
     for i in range(3):
         e2e_step(i)
+    e2e_join()
     torch.cuda.synchronize()
     multi.barrier()
     ev0.record(stream)
     for i in range(e2e_steps):
         e2e_step(i)
+    e2e_join()
     ev1.record(stream)
     torch.cuda.synchronize()
     multi.barrier()

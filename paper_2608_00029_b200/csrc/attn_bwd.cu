@@ -494,12 +494,10 @@ __device__ __forceinline__ void bwd_compute(uint8_t* smem, BwdBars* bars, uint32
 
             // ---- dS phase: ds = p * (dp - delta); bf16 to TMEM (for dK) and to swizzled smem (for dQ).
             // p is taken from the bf16 pairs already in registers.
+            // dP^T of this tile was queued after dQ of the previous one and the tensor pipe completes in
+            // order, so this wait also covers "the previous dQ has finished reading the dS staging buffer".
             ok = mbar_wait(&bars->dp_full, g & 1, abort_flag);
             if (!ok) break;
-            if (g > 0) {  // the dQ UMMA of the previous tile must be done reading the dS staging buffer
-                ok = mbar_wait(&bars->dq_full, (g - 1) & 1, abort_flag);
-                if (!ok) break;
-            }
             tc_fence_after();
             uint32_t dd[32];
             {
