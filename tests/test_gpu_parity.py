@@ -126,6 +126,27 @@ def test_edge_shapes(B, H, T, D, causal):
         assert got["dQ"].float().abs().max() < 1e-5 and got["dK"].float().abs().max() < 1e-5
 
 
+GRID = [  # (B, H, T, D, causal, sampled heads): corners of the paper's benchmark ranges, at its batch of 16
+    (16, 32, 2048, 128, True, 2),
+    (16, 32, 512, 128, True, 3),
+    (16, 20, 1024, 64, True, 3),
+    (16, 12, 2048, 64, False, 2),
+]
+
+
+@pytest.mark.parametrize("B,H,T,D,causal,n_heads", GRID)
+def test_benchmark_grid_shapes(B, H, T, D, causal, n_heads):
+    """Shapes from the ranges of the paper's attention microbenchmark (sequence lengths 512 to 2048, 12 to
+    32 heads, head dimension 64 or 128), run at full size on the GPU and compared on sampled heads."""
+    h = _harness()
+    cfg = W.AttnConfig(f"grid_{T}_{H}_{D}", B=B, H=H, T=T, D=D, seed=300 + T + H + D, causal=causal)
+    Q, K, V, dO = W.make_inputs(cfg)
+    got = h.run_gpu(Q, K, V, dO, cfg.scale, causal)
+    heads = sorted({((i * 7 + 3) % B, (i * 11 + 5) % H) for i in range(n_heads)})
+    ref = h.run_oracle(Q, K, V, dO, cfg.scale, causal, heads=heads)
+    h.compare(h.select_heads(got, heads), ref, label=f"grid T={T} H={H} D={D} causal={causal}: ", dO=ref["dO_in"])
+
+
 def test_peaked_softmax_large_scores():
     """Scores ~ N(0, 16^2) (Q, K ~ 4 N(0,1)): exercises the running-max rescale and the exp range far
     beyond the five configurations.  |K| and |dS| are 4x and ~10x larger than there, and dQ, dK are sums
