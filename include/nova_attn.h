@@ -161,6 +161,44 @@ int nova_attn_bwd_static_scratch(const void* Q, const void* K, const void* V, co
                                  void* dQ, void* dK, void* dV, int B, int H, int T, int D,
                                  float scale, int causal, void* stream);
 
+/*
+ * Strided variants (paper Section 4.2: the per-head layout change around attention is expressed in the
+ * access pattern, so the transposes between the fused projection output and the per-head tensors cost
+ * nothing).  Each bf16 tensor is addressed as element (b, h, t, d) at
+ *     base + b * batch + h * head + t * token + d          (strides in ELEMENTS, d contiguous),
+ * so Q, K and V can be read straight out of a fused projection output [B, T, 3, H, D]
+ * (Q: base + 0, K: base + H*D, V: base + 2*H*D, each with batch = T*3*H*D, head = D, token = 3*H*D) and
+ * O, dQ, dK, dV written as [B, T, H, D] (batch = T*H*D, head = D, token = H*D), or any other layout with
+ *   - every stride a multiple of 8 elements (16 bytes; NOVA_ATTN_ERR_ALIGNMENT otherwise),
+ *   - token >= D, head >= 8, batch >= 8, every stride below 2^39 (NOVA_ATTN_ERR_SHAPE otherwise),
+ *   - strides that the TMA descriptor encoder accepts once token / head / batch are sorted by stride (it
+ *     rejects, with NOVA_ATTN_ERR_CUDA, layouts whose larger strides are not multiples it can express),
+ *   - no two elements of an OUTPUT tensor at the same address, outputs not overlapping inputs.
+ * LSE and Delta stay contiguous fp32 [B, H, T].  Everything else (shapes, validation, results, errors,
+ * workspace) is as for nova_attn_fwd, nova_attn_bwd_preprocess and nova_attn_bwd; those three are the
+ * special case batch = H*T*D, head = T*D, token = D.  nova_attn_bwd_strided takes no O (Delta carries it).
+ */
+typedef struct nova_attn_strides {
+    long long batch, head, token;
+} nova_attn_strides;
+
+int nova_attn_fwd_strided(const void* Q, const void* K, const void* V, void* O, float* LSE,
+                          int B, int H, int T, int D,
+                          const nova_attn_strides* q_strides, const nova_attn_strides* k_strides,
+                          const nova_attn_strides* v_strides, const nova_attn_strides* o_strides,
+                          float scale, int causal, void* stream);
+int nova_attn_bwd_preprocess_strided(const void* O, const void* dO, float* Delta, int B, int H, int T, int D,
+                                     const nova_attn_strides* o_strides, const nova_attn_strides* do_strides,
+                                     void* stream);
+int nova_attn_bwd_strided(const void* Q, const void* K, const void* V, const void* dO,
+                          const float* LSE, const float* Delta, void* dQ, void* dK, void* dV,
+                          int B, int H, int T, int D,
+                          const nova_attn_strides* q_strides, const nova_attn_strides* k_strides,
+                          const nova_attn_strides* v_strides, const nova_attn_strides* do_strides,
+                          const nova_attn_strides* dq_strides, const nova_attn_strides* dk_strides,
+                          const nova_attn_strides* dv_strides,
+                          float scale, int causal, void* workspace, size_t workspace_bytes, void* stream);
+
 /* Static, never-freed description of a status code. */
 const char* nova_attn_status_string(int status);
 

@@ -78,11 +78,12 @@ int device_state(DeviceState** out) {
     return NOVA_ATTN_OK;
 }
 
-// Tensor maps are pure functions of (pointer, D, T, B*H); a small cache keeps the host cost of a
+// Tensor maps are pure functions of (pointer, shape, strides); a small cache keeps the host cost of a
 // call to a lookup when the same buffers are used step after step.
 struct MapKey {
     const void* ptr;
     int D, T, BH, dev, elem_bytes;
+    long long st, sh;
 };
 struct MapEntry {
     MapKey key{};
@@ -92,22 +93,27 @@ struct MapEntry {
 constexpr int kMapCache = 128;
 MapEntry g_maps[kMapCache];
 
+// 3-D map [D, T, B*H] of a tensor whose heads and batches merge into one dimension of stride `sh`
+// elements (0: contiguous, sh = T*D) with token stride `st` (0: D).
 // elem_bytes 2: bf16 tensor, box [64, 128, 1]; elem_bytes 4: fp32 tensor, box [32, 128, 1].
-int get_tensor_map(const void* ptr, int D, long long T, long long BH, CUtensorMap* out, int elem_bytes = 2) {
+int get_tensor_map(const void* ptr, int D, long long T, long long BH, CUtensorMap* out, int elem_bytes = 2,
+                   long long st = 0, long long sh = 0) {
     int dev = 0;
     cudaGetDevice(&dev);
-    const MapKey key{ptr, D, static_cast<int>(T), static_cast<int>(BH), dev, elem_bytes};
+    if (st == 0) st = D;
+    if (sh == 0) sh = T * D;
+    const MapKey key{ptr, D, static_cast<int>(T), static_cast<int>(BH), dev, elem_bytes, st, sh};
     const uint64_t h = (reinterpret_cast<uint64_t>(ptr) >> 8) * 0x9E3779B97F4A7C15ull + uint64_t(T) * 31 + uint64_t(BH) * 131 + D;
     std::lock_guard<std::mutex> lock(g_mutex);
     MapEntry& e = g_maps[(h >> 32) % kMapCache];
     if (e.valid && e.key.ptr == key.ptr && e.key.D == key.D && e.key.T == key.T && e.key.BH == key.BH &&
-        e.key.dev == key.dev && e.key.elem_bytes == key.elem_bytes) {
+        e.key.dev == key.dev && e.key.elem_bytes == key.elem_bytes && e.key.st == key.st && e.key.sh == key.sh) {
         *out = e.map;
         return NOVA_ATTN_OK;
     }
     // [D, T, B*H], D contiguous; 128-byte box rows; rows past T read as zero and are clipped on writes.
     const cuuint64_t dims[3] = {cuuint64_t(D), cuuint64_t(T), cuuint64_t(BH)};
-    const cuuint64_t strides[2] = {cuuint64_t(D) * elem_bytes, cuuint64_t(T) * cuuint64_t(D) * elem_bytes};
+    const cuuint64_t strides[2] = {cuuint64_t(st) * elem_bytes, cuuint64_t(sh) * elem_bytes};
     const cuuint32_t box[3] = {cuuint32_t(128 / elem_bytes), cuuint32_t(kBlockQ), 1};
     const cuuint32_t estr[3] = {1, 1, 1};
     CUtensorMap m;
@@ -120,6 +126,100 @@ int get_tensor_map(const void* ptr, int D, long long T, long long BH, CUtensorMa
     e.map = m;
     e.valid = true;
     *out = m;
+    return NOVA_ATTN_OK;
+}
+
+// 4-D map of a bf16 tensor indexed [b, h, t, d] with strides `st` (elements): dimensions [D, x, y, z] where
+// x, y, z are token / head / batch in order of increasing stride (the encoder wants that), box 64 x 128
+// tokens.  `*order` receives which of the three sits where (the code tma_order_coords understands).
+struct Map4Key {
+    const void* ptr;
+    int D, T, H, B, dev;
+    long long sb, sh, st;
+};
+struct Map4Entry {
+    Map4Key key{};
+    bool valid = false;
+    int order = 0;
+    CUtensorMap map;
+};
+Map4Entry g_maps4[kMapCache];
+
+int get_tensor_map4(const void* ptr, const AttnShape& s, const TensorStrides& st, CUtensorMap* out, uint32_t* order) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    const Map4Key key{ptr, s.D, s.T, s.H, s.B, dev, st.b, st.h, st.t};
+    const uint64_t h = (reinterpret_cast<uint64_t>(ptr) >> 8) * 0x9E3779B97F4A7C15ull + uint64_t(s.T) * 31 +
+                       uint64_t(s.B) * 131 + uint64_t(s.H) * 17 + uint64_t(st.t) * 7 + s.D;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    Map4Entry& e = g_maps4[(h >> 32) % kMapCache];
+    if (e.valid && e.key.ptr == key.ptr && e.key.D == key.D && e.key.T == key.T && e.key.H == key.H &&
+        e.key.B == key.B && e.key.dev == key.dev && e.key.sb == key.sb && e.key.sh == key.sh && e.key.st == key.st) {
+        *out = e.map;
+        *order = static_cast<uint32_t>(e.order);
+        return NOVA_ATTN_OK;
+    }
+    // which: 0 = token, 1 = head, 2 = batch; sorted by stride (ties keep token < head < batch)
+    int which[3] = {0, 1, 2};
+    const long long stride_of[3] = {st.t, st.h, st.b};
+    const int extent_of[3] = {s.T, s.H, s.B};
+    for (int i = 1; i < 3; ++i)
+        for (int j = i; j > 0 && stride_of[which[j]] < stride_of[which[j - 1]]; --j) {
+            const int tmp = which[j];
+            which[j] = which[j - 1];
+            which[j - 1] = tmp;
+        }
+    static const int kCodes[3][3] = {{-1, 0, 2}, {1, -1, 4}, {3, 5, -1}};  // [which[0]][which[1]] -> order code
+    const int code = kCodes[which[0]][which[1]];
+    cuuint64_t dims[4] = {cuuint64_t(s.D), 0, 0, 0};
+    cuuint64_t strides[3];
+    cuuint32_t box[4] = {cuuint32_t(kBoxCols), 1, 1, 1};
+    for (int i = 0; i < 3; ++i) {
+        dims[1 + i] = cuuint64_t(extent_of[which[i]]);
+        strides[i] = cuuint64_t(stride_of[which[i]]) * sizeof(__nv_bfloat16);
+        if (which[i] == 0) box[1 + i] = cuuint32_t(kBlockQ);
+    }
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUtensorMap m;
+    const CUresult r = g_encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), dims, strides, box, estr,
+                                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail_cuda(static_cast<int>(r));
+    e.key = key;
+    e.map = m;
+    e.order = code;
+    e.valid = true;
+    *out = m;
+    *order = static_cast<uint32_t>(code);
+    return NOVA_ATTN_OK;
+}
+
+// Heads and batches of the tensor merge into one dimension (the [B,H,T,D] family): 3-D maps, plain kernels.
+bool merges(const AttnShape& s, const TensorStrides& st) {
+    return st.b == static_cast<long long>(s.H) * st.h && st.t <= st.h;
+}
+
+// The map of a bf16 tensor for the plain (3-D) or the strided (4-D) build of the kernels.
+int get_bf16_map(const void* ptr, const AttnShape& s, const TensorStrides& st, bool strided, CUtensorMap* out,
+                 uint32_t* order) {
+    if (strided) return get_tensor_map4(ptr, s, st, out, order);
+    *order = 0;
+    return get_tensor_map(ptr, s.D, s.T, static_cast<long long>(s.B) * s.H, out, 2, st.t, st.h);
+}
+
+TensorStrides contiguous_strides(int H, int T, int D) {
+    return TensorStrides{static_cast<long long>(H) * T * D, static_cast<long long>(T) * D, static_cast<long long>(D)};
+}
+
+// Strides are in elements; every one a multiple of 8 (16 bytes, which TMA and the 16-byte accesses of the
+// helper kernels need), the token stride at least D, none so large that a byte offset leaves 2^40.
+int check_strides(const nova_attn_strides* p, int D, TensorStrides* out) {
+    if (!p) return NOVA_ATTN_ERR_NULL;
+    if ((p->batch & 7) || (p->head & 7) || (p->token & 7)) return NOVA_ATTN_ERR_ALIGNMENT;
+    if (p->token < D || p->head < 8 || p->batch < 8) return NOVA_ATTN_ERR_SHAPE;
+    const long long lim = (1ll << 39);
+    if (p->token >= lim || p->head >= lim || p->batch >= lim) return NOVA_ATTN_ERR_SHAPE;
+    *out = TensorStrides{p->batch, p->head, p->token};
     return NOVA_ATTN_OK;
 }
 
@@ -148,37 +248,66 @@ using namespace nova;
 
 extern "C" {
 
-int nova_attn_fwd(const void* Q, const void* K, const void* V, void* O, float* LSE, int B, int H, int T, int D,
-                  float scale, int causal, void* stream) {
+int nova_attn_fwd_strided(const void* Q, const void* K, const void* V, void* O, float* LSE, int B, int H, int T, int D,
+                          const nova_attn_strides* q_strides, const nova_attn_strides* k_strides,
+                          const nova_attn_strides* v_strides, const nova_attn_strides* o_strides, float scale,
+                          int causal, void* stream) {
     if (!Q || !K || !V || !O || !LSE) return NOVA_ATTN_ERR_NULL;
     if (int rc = check_shape(B, H, T, D)) return rc;
     if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(LSE)) return NOVA_ATTN_ERR_ALIGNMENT;
     if (!std::isfinite(scale) || !(scale > 0.f)) return NOVA_ATTN_ERR_SCALE;
+    TensorStrides sq, sk, sv, so;
+    if (int rc = check_strides(q_strides, D, &sq)) return rc;
+    if (int rc = check_strides(k_strides, D, &sk)) return rc;
+    if (int rc = check_strides(v_strides, D, &sv)) return rc;
+    if (int rc = check_strides(o_strides, D, &so)) return rc;
     DeviceState* st = nullptr;
     if (int rc = device_state(&st)) return rc;
-    const long long BH = static_cast<long long>(B) * H;
-    CUtensorMap tmQ, tmK, tmV, tmO;
-    if (int rc = get_tensor_map(Q, D, T, BH, &tmQ)) return rc;
-    if (int rc = get_tensor_map(K, D, T, BH, &tmK)) return rc;
-    if (int rc = get_tensor_map(V, D, T, BH, &tmV)) return rc;
-    if (int rc = get_tensor_map(O, D, T, BH, &tmO)) return rc;
     const AttnShape s{B, H, T, D, causal != 0, scale};
-    const cudaError_t e = launch_attn_fwd(tmQ, tmK, tmV, tmO, LSE, s, st->num_sms, st->dev_status,
+    CUtensorMap tmQ, tmK, tmV, tmO;
+    uint32_t oq, ok, ov, oo;
+    const bool strided = !(merges(s, sq) && merges(s, sk) && merges(s, sv) && merges(s, so));
+    if (int rc = get_bf16_map(Q, s, sq, strided, &tmQ, &oq)) return rc;
+    if (int rc = get_bf16_map(K, s, sk, strided, &tmK, &ok)) return rc;
+    if (int rc = get_bf16_map(V, s, sv, strided, &tmV, &ov)) return rc;
+    if (int rc = get_bf16_map(O, s, so, strided, &tmO, &oo)) return rc;
+    const uint32_t orders = oq | (ok << 4) | (ov << 8) | (oo << 12);
+    const cudaError_t e = launch_attn_fwd(tmQ, tmK, tmV, tmO, strided, orders, LSE, s, st->num_sms, st->dev_status,
                                           static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? NOVA_ATTN_OK : fail_cuda(e);
 }
 
-int nova_attn_bwd_preprocess(const void* O, const void* dO, float* Delta, int B, int H, int T, int D, void* stream) {
+int nova_attn_fwd(const void* Q, const void* K, const void* V, void* O, float* LSE, int B, int H, int T, int D,
+                  float scale, int causal, void* stream) {
+    if (int rc = check_shape(B, H, T, D)) return rc;
+    const TensorStrides c = contiguous_strides(H, T, D);
+    const nova_attn_strides n{c.b, c.h, c.t};
+    return nova_attn_fwd_strided(Q, K, V, O, LSE, B, H, T, D, &n, &n, &n, &n, scale, causal, stream);
+}
+
+int nova_attn_bwd_preprocess_strided(const void* O, const void* dO, float* Delta, int B, int H, int T, int D,
+                                     const nova_attn_strides* o_strides, const nova_attn_strides* do_strides,
+                                     void* stream) {
     if (!O || !dO || !Delta) return NOVA_ATTN_ERR_NULL;
     if (int rc = check_shape(B, H, T, D)) return rc;
     if (!aligned16(O) || !aligned16(dO) || !aligned16(Delta)) return NOVA_ATTN_ERR_ALIGNMENT;
+    TensorStrides so, sdo;
+    if (int rc = check_strides(o_strides, D, &so)) return rc;
+    if (int rc = check_strides(do_strides, D, &sdo)) return rc;
     DeviceState* st = nullptr;
     if (int rc = device_state(&st)) return rc;
-    const long long rows = static_cast<long long>(B) * H * T;
+    const AttnShape s{B, H, T, D, 1, 1.f};
     const cudaError_t e =
-        launch_attn_bwd_preprocess(static_cast<const __nv_bfloat16*>(O), static_cast<const __nv_bfloat16*>(dO), Delta,
-                                   rows, D, st->num_sms, static_cast<cudaStream_t>(stream));
+        launch_attn_bwd_preprocess(static_cast<const __nv_bfloat16*>(O), static_cast<const __nv_bfloat16*>(dO), Delta, s,
+                                   so, sdo, st->num_sms, static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? NOVA_ATTN_OK : fail_cuda(e);
+}
+
+int nova_attn_bwd_preprocess(const void* O, const void* dO, float* Delta, int B, int H, int T, int D, void* stream) {
+    if (int rc = check_shape(B, H, T, D)) return rc;
+    const TensorStrides c = contiguous_strides(H, T, D);
+    const nova_attn_strides n{c.b, c.h, c.t};
+    return nova_attn_bwd_preprocess_strided(O, dO, Delta, B, H, T, D, &n, &n, stream);
 }
 
 int nova_attn_bwd_preprocess_exact(const void* Q, const void* K, const void* V, const void* dO, const float* LSE,
@@ -207,10 +336,13 @@ size_t nova_attn_bwd_workspace_bytes(int B, int H, int T, int D) {
     return acc_bytes(B, H, T, D);
 }
 
-int nova_attn_bwd_steps(const void* Q, const void* K, const void* V, const void* O, const void* dO, const float* LSE,
-                        const float* Delta, void* dQ, void* dK, void* dV, int B, int H, int T, int D, float scale,
-                        int causal, void* workspace, size_t workspace_bytes, void* stream, int steps) {
-    (void)O;  // Delta already carries rowsum(dO * O)
+namespace {
+// The three steps of the backward on strided bf16 tensors; `steps` as in nova_attn_bwd_steps.
+int bwd_impl(const void* Q, const void* K, const void* V, const void* dO, const float* LSE, const float* Delta, void* dQ,
+             void* dK, void* dV, int B, int H, int T, int D, const TensorStrides& sq, const TensorStrides& sk,
+             const TensorStrides& sv, const TensorStrides& sdo, const TensorStrides& sdq, const TensorStrides& sdk,
+             const TensorStrides& sdv, float scale, int causal, void* workspace, size_t workspace_bytes, void* stream,
+             int steps) {
     if (!Q || !K || !V || !dO || !LSE || !Delta || !dQ || !dK || !dV) return NOVA_ATTN_ERR_NULL;
     if (int rc = check_shape(B, H, T, D)) return rc;
     if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(dO) || !aligned16(LSE) || !aligned16(Delta) ||
@@ -225,6 +357,7 @@ int nova_attn_bwd_steps(const void* Q, const void* K, const void* V, const void*
     const long long BH = static_cast<long long>(B) * H;
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     float* acc = static_cast<float*>(workspace);
+    const AttnShape s{B, H, T, D, causal != 0, scale};
     cudaError_t e = cudaSuccess;
     if (steps & NOVA_ATTN_BWD_STEP_ZERO) {
         e = launch_zero(acc, need, st->num_sms, cs);
@@ -232,24 +365,37 @@ int nova_attn_bwd_steps(const void* Q, const void* K, const void* V, const void*
     }
     if (steps & NOVA_ATTN_BWD_STEP_MAIN) {
         CUtensorMap tmQ, tmK, tmV, tmdO, tmAcc, tmdK, tmdV;
-        if (int rc = get_tensor_map(Q, D, T, BH, &tmQ)) return rc;
-        if (int rc = get_tensor_map(K, D, T, BH, &tmK)) return rc;
-        if (int rc = get_tensor_map(V, D, T, BH, &tmV)) return rc;
-        if (int rc = get_tensor_map(dO, D, T, BH, &tmdO)) return rc;
+        uint32_t oq, ok, ov, odo, odk, odv;
+        const bool strided = !(merges(s, sq) && merges(s, sk) && merges(s, sv) && merges(s, sdo) && merges(s, sdk) &&
+                               merges(s, sdv));
+        if (int rc = get_bf16_map(Q, s, sq, strided, &tmQ, &oq)) return rc;
+        if (int rc = get_bf16_map(K, s, sk, strided, &tmK, &ok)) return rc;
+        if (int rc = get_bf16_map(V, s, sv, strided, &tmV, &ov)) return rc;
+        if (int rc = get_bf16_map(dO, s, sdo, strided, &tmdO, &odo)) return rc;
         if (int rc = get_tensor_map(acc, D, T, BH, &tmAcc, 4)) return rc;
-        if (int rc = get_tensor_map(dK, D, T, BH, &tmdK)) return rc;
-        if (int rc = get_tensor_map(dV, D, T, BH, &tmdV)) return rc;
-        const AttnShape s{B, H, T, D, causal != 0, scale};
-        e = launch_attn_bwd(tmQ, tmK, tmV, tmdO, tmAcc, tmdK, tmdV, LSE, Delta, static_cast<__nv_bfloat16*>(dK),
-                            static_cast<__nv_bfloat16*>(dV), s, st->num_sms, st->dev_status, cs);
+        if (int rc = get_bf16_map(dK, s, sdk, strided, &tmdK, &odk)) return rc;
+        if (int rc = get_bf16_map(dV, s, sdv, strided, &tmdV, &odv)) return rc;
+        const uint32_t orders = oq | (ok << 4) | (ov << 8) | (odo << 12) | (odk << 16) | (odv << 20);
+        e = launch_attn_bwd(tmQ, tmK, tmV, tmdO, tmAcc, tmdK, tmdV, strided, orders, LSE, Delta, static_cast<__nv_bfloat16*>(dK),
+                            static_cast<__nv_bfloat16*>(dV), sdk, sdv, s, st->num_sms, st->dev_status, cs);
         if (e != cudaSuccess) return fail_cuda(e);
     }
     if (steps & NOVA_ATTN_BWD_STEP_CONVERT) {
-        e = launch_dq_convert(acc, static_cast<__nv_bfloat16*>(dQ), static_cast<long long>(B) * H * T * D, scale,
-                              st->num_sms, cs);
+        e = launch_dq_convert(acc, static_cast<__nv_bfloat16*>(dQ), s, sdq, scale, st->num_sms, cs);
         if (e != cudaSuccess) return fail_cuda(e);
     }
     return NOVA_ATTN_OK;
+}
+}  // namespace
+
+int nova_attn_bwd_steps(const void* Q, const void* K, const void* V, const void* O, const void* dO, const float* LSE,
+                        const float* Delta, void* dQ, void* dK, void* dV, int B, int H, int T, int D, float scale,
+                        int causal, void* workspace, size_t workspace_bytes, void* stream, int steps) {
+    (void)O;  // Delta already carries rowsum(dO * O)
+    if (int rc = check_shape(B, H, T, D)) return rc;
+    const TensorStrides c = contiguous_strides(H, T, D);
+    return bwd_impl(Q, K, V, dO, LSE, Delta, dQ, dK, dV, B, H, T, D, c, c, c, c, c, c, c, scale, causal, workspace,
+                    workspace_bytes, stream, steps);
 }
 
 int nova_attn_bwd(const void* Q, const void* K, const void* V, const void* O, const void* dO, const float* LSE,
@@ -258,6 +404,27 @@ int nova_attn_bwd(const void* Q, const void* K, const void* V, const void* O, co
     return nova_attn_bwd_steps(Q, K, V, O, dO, LSE, Delta, dQ, dK, dV, B, H, T, D, scale, causal, workspace,
                                workspace_bytes, stream,
                                NOVA_ATTN_BWD_STEP_ZERO | NOVA_ATTN_BWD_STEP_MAIN | NOVA_ATTN_BWD_STEP_CONVERT);
+}
+
+int nova_attn_bwd_strided(const void* Q, const void* K, const void* V, const void* dO, const float* LSE,
+                          const float* Delta, void* dQ, void* dK, void* dV, int B, int H, int T, int D,
+                          const nova_attn_strides* q_strides, const nova_attn_strides* k_strides,
+                          const nova_attn_strides* v_strides, const nova_attn_strides* do_strides,
+                          const nova_attn_strides* dq_strides, const nova_attn_strides* dk_strides,
+                          const nova_attn_strides* dv_strides, float scale, int causal, void* workspace,
+                          size_t workspace_bytes, void* stream) {
+    if (int rc = check_shape(B, H, T, D)) return rc;
+    TensorStrides sq, sk, sv, sdo, sdq, sdk, sdv;
+    if (int rc = check_strides(q_strides, D, &sq)) return rc;
+    if (int rc = check_strides(k_strides, D, &sk)) return rc;
+    if (int rc = check_strides(v_strides, D, &sv)) return rc;
+    if (int rc = check_strides(do_strides, D, &sdo)) return rc;
+    if (int rc = check_strides(dq_strides, D, &sdq)) return rc;
+    if (int rc = check_strides(dk_strides, D, &sdk)) return rc;
+    if (int rc = check_strides(dv_strides, D, &sdv)) return rc;
+    return bwd_impl(Q, K, V, dO, LSE, Delta, dQ, dK, dV, B, H, T, D, sq, sk, sv, sdo, sdq, sdk, sdv, scale, causal,
+                    workspace, workspace_bytes, stream,
+                    NOVA_ATTN_BWD_STEP_ZERO | NOVA_ATTN_BWD_STEP_MAIN | NOVA_ATTN_BWD_STEP_CONVERT);
 }
 
 const char* nova_attn_status_string(int status) {

@@ -103,7 +103,8 @@ struct BwdBars {
 // This CTA's list of work items.  Items are ordered by weight (key tile 0 of a causal problem sees
 // every query tile, the last key tile only one) and dealt to the CTAs in zig-zag passes.
 struct WorkList {
-    int n_items, n_ctas, cta, BH, n_tiles;
+    int n_items, n_ctas, cta, BH, n_tiles, H;
+    uint32_t orders;  // coordinate orders of the Q, K, V, dO, dK, dV tensor maps, four bits each
     bool causal;
     __device__ __forceinline__ int passes() const { return (n_items + n_ctas - 1) / n_ctas; }
     // Item of pass p: returns false if this CTA has none in that pass.
@@ -118,7 +119,7 @@ struct WorkList {
     }
 };
 
-template <int D>
+template <int D, bool kStrided>
 __device__ __forceinline__ void bwd_producer(const CUtensorMap* tmQ, const CUtensorMap* tmK, const CUtensorMap* tmV,
                                              const CUtensorMap* tmdO, uint8_t* smem, BwdBars* bars,
                                              const WorkList& wl) {
@@ -130,6 +131,7 @@ __device__ __forceinline__ void bwd_producer(const CUtensorMap* tmQ, const CUten
     for (int p = 0; p < wl.passes() && ok; ++p) {
         int kt, bh, i0, n_it;
         if (!wl.get(p, &kt, &bh, &i0, &n_it)) continue;
+        const int head = kStrided ? bh % wl.H : 0, batch = kStrided ? bh / wl.H : 0;
         const int ks = w % Cfg::kKVStages;
         const uint32_t kph = (w / Cfg::kKVStages) & 1;
         ok = mbar_wait(&bars->kv_empty[ks], kph ^ 1, abort_flag);
@@ -138,10 +140,10 @@ __device__ __forceinline__ void bwd_producer(const CUtensorMap* tmQ, const CUten
         armed_kv[ks] = kph;
 #pragma unroll
         for (int h = 0; h < Cfg::kHalves; ++h) {
-            tma_load_3d(smem + Cfg::kOffK + ks * Cfg::kTileBytes + h * kHalfTileBytes, tmK, &bars->kv_full[ks],
-                        h * kBoxCols, kt * kBlockK, bh);
-            tma_load_3d(smem + Cfg::kOffV + ks * Cfg::kTileBytes + h * kHalfTileBytes, tmV, &bars->kv_full[ks],
-                        h * kBoxCols, kt * kBlockK, bh);
+            tma_load_tile<kStrided>(smem + Cfg::kOffK + ks * Cfg::kTileBytes + h * kHalfTileBytes, tmK, &bars->kv_full[ks],
+                          (wl.orders >> 4) & 15, h * kBoxCols, kt * kBlockK, head, batch, bh);
+            tma_load_tile<kStrided>(smem + Cfg::kOffV + ks * Cfg::kTileBytes + h * kHalfTileBytes, tmV, &bars->kv_full[ks],
+                          (wl.orders >> 8) & 15, h * kBoxCols, kt * kBlockK, head, batch, bh);
         }
         for (int it = 0; it < n_it; ++it, ++g) {
             const int st = g & 1;
@@ -152,8 +154,8 @@ __device__ __forceinline__ void bwd_producer(const CUtensorMap* tmQ, const CUten
             armed_q[st] = (g >> 1) & 1;
 #pragma unroll
             for (int h = 0; h < Cfg::kHalves; ++h)
-                tma_load_3d(smem + Cfg::kOffQ + st * Cfg::kTileBytes + h * kHalfTileBytes, tmQ, &bars->q_full[st],
-                            h * kBoxCols, qrow, bh);
+                tma_load_tile<kStrided>(smem + Cfg::kOffQ + st * Cfg::kTileBytes + h * kHalfTileBytes, tmQ, &bars->q_full[st],
+                              wl.orders & 15, h * kBoxCols, qrow, head, batch, bh);
             const int ds = g % Cfg::kdOStages;
             const uint32_t dph = (g / Cfg::kdOStages) & 1;
             ok = mbar_wait(&bars->do_empty[ds], dph ^ 1, abort_flag);
@@ -162,8 +164,8 @@ __device__ __forceinline__ void bwd_producer(const CUtensorMap* tmQ, const CUten
             armed_do[ds] = dph;
 #pragma unroll
             for (int h = 0; h < Cfg::kHalves; ++h)
-                tma_load_3d(smem + Cfg::kOffdO + ds * Cfg::kTileBytes + h * kHalfTileBytes, tmdO, &bars->do_full[ds],
-                            h * kBoxCols, qrow, bh);
+                tma_load_tile<kStrided>(smem + Cfg::kOffdO + ds * Cfg::kTileBytes + h * kHalfTileBytes, tmdO, &bars->do_full[ds],
+                              (wl.orders >> 12) & 15, h * kBoxCols, qrow, head, batch, bh);
         }
         ++w;
     }
@@ -434,8 +436,9 @@ __device__ __forceinline__ void bwd_store_dkv32(const uint32_t (&a)[32], const u
 
 template <int D, bool kCausal>
 __device__ __forceinline__ void bwd_compute(uint8_t* smem, BwdBars* bars, uint32_t tmem_base,
-                                            __nv_bfloat16* __restrict__ dK, __nv_bfloat16* __restrict__ dV, int T,
-                                            float scale, const WorkList& wl, int cwarp, int lane) {
+                                            __nv_bfloat16* __restrict__ dK, __nv_bfloat16* __restrict__ dV,
+                                            const TensorStrides& sdk, const TensorStrides& sdv, int T, float scale,
+                                            const WorkList& wl, int cwarp, int lane) {
     using Cfg = BwdCfg<D>;
     volatile int* abort_flag = &bars->abort_flag;
     const uint32_t lane_base = 32u * (cwarp & 3);
@@ -547,9 +550,9 @@ __device__ __forceinline__ void bwd_compute(uint8_t* smem, BwdBars* bars, uint32
             ok = mbar_wait(&bars->dkv_full, w & 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
-            const size_t out_off = (static_cast<size_t>(bh) * T + key) * D + half * kColsPerThread;
-            uint4* dv_row = reinterpret_cast<uint4*>(dV + out_off);
-            uint4* dk_row = reinterpret_cast<uint4*>(dK + out_off);
+            const long long hb = bh % wl.H, bb = bh / wl.H;
+            uint4* dv_row = reinterpret_cast<uint4*>(dV + bb * sdv.b + hb * sdv.h + key * sdv.t + half * kColsPerThread);
+            uint4* dk_row = reinterpret_cast<uint4*>(dK + bb * sdk.b + hb * sdk.h + key * sdk.t + half * kColsPerThread);
 #pragma unroll
             for (int cb = 0; cb < kColsPerThread; cb += 32) {
                 uint32_t a[32], bq[32];
@@ -573,6 +576,7 @@ __device__ __forceinline__ void bwd_compute(uint8_t* smem, BwdBars* bars, uint32
 // warps move on to the next item at once.  Nothing waits for a reduction or a store to complete
 // except the end of the kernel; before the staging buffer is refilled, the leader checks that the copy
 // engine has read it.
+template <bool kStrided>
 __device__ __forceinline__ void bwd_dq_tma(uint8_t* smem, BwdBars* bars, uint32_t tmem_base, const CUtensorMap* tmAcc,
                                            const CUtensorMap* tmdK, const CUtensorMap* tmdV, float scale,
                                            const WorkList& wl, int qwarp, int lane) {
@@ -606,8 +610,9 @@ __device__ __forceinline__ void bwd_dq_tma(uint8_t* smem, BwdBars* bars, uint32_
                     tma_reduce_add_3d(tmAcc, stage, 0, row, bh);
                     tma_reduce_add_3d(tmAcc, stage + kHalfTileBytes, 32, row, bh);
                 } else {
-                    tma_store_3d(tmdV, stage, 0, row, bh);
-                    tma_store_3d(tmdK, stage + kHalfTileBytes, 0, row, bh);
+                    const int hh = kStrided ? bh % wl.H : 0, bb = kStrided ? bh / wl.H : 0;
+                    tma_store_tile<kStrided>(tmdV, stage, (wl.orders >> 20) & 15, 0, row, hh, bb, bh);
+                    tma_store_tile<kStrided>(tmdK, stage + kHalfTileBytes, (wl.orders >> 16) & 15, 0, row, hh, bb, bh);
                 }
                 bulk_commit_group();
             }
@@ -777,15 +782,15 @@ __device__ __forceinline__ void bwd_dq_tma_wide(uint8_t* smem, BwdBars* bars, ui
     if (leader) bulk_wait_group<0>();
 }
 
-template <int D, bool kCausal>
+template <int D, bool kCausal, bool kStrided>
 __global__ void __launch_bounds__(kBwdThreads, 1)
 attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmdO,
                 const __grid_constant__ CUtensorMap tmAcc, const __grid_constant__ CUtensorMap tmdK,
                 const __grid_constant__ CUtensorMap tmdV, const float* __restrict__ LSE,
                 const float* __restrict__ Delta, __nv_bfloat16* __restrict__ dK,
-                __nv_bfloat16* __restrict__ dV, int T, int BH, int n_tiles, float scale,
-                int* __restrict__ dev_status) {
+                __nv_bfloat16* __restrict__ dV, const TensorStrides sdk, const TensorStrides sdv, int T, int BH,
+                int H, uint32_t orders, int n_tiles, float scale, int* __restrict__ dev_status) {
     using Cfg = BwdCfg<D>;
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -795,7 +800,8 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     }
     BwdBars* bars = reinterpret_cast<BwdBars*>(smem + Cfg::kOffBar);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const WorkList wl{n_tiles * BH, static_cast<int>(gridDim.x), static_cast<int>(blockIdx.x), BH, n_tiles, kCausal};
+    const WorkList wl{n_tiles * BH, static_cast<int>(gridDim.x), static_cast<int>(blockIdx.x), BH, n_tiles, H, orders,
+                      kCausal};
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < 2; ++s) {
@@ -841,16 +847,16 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     griddep_wait();  // everything above overlaps the previous kernel of the stream
 
     if (warp == 0) {
-        if (lane == 0) bwd_producer<D>(&tmQ, &tmK, &tmV, &tmdO, smem, bars, wl);
+        if (lane == 0) bwd_producer<D, kStrided>(&tmQ, &tmK, &tmV, &tmdO, smem, bars, wl);
     } else if (warp == 1) {
         bwd_mma<D>(smem, bars, tmem_base, wl);
     } else if (warp < 4) {
         bwd_rows(bars, reinterpret_cast<float*>(smem + Cfg::kOffRow), LSE, Delta, T, wl, (warp - 2) * 32 + lane);
     } else if (warp < 12) {
-        bwd_compute<D, kCausal>(smem, bars, tmem_base, dK, dV, T, scale, wl, warp - 4, lane);
+        bwd_compute<D, kCausal>(smem, bars, tmem_base, dK, dV, sdk, sdv, T, scale, wl, warp - 4, lane);
     } else {
         if constexpr (Cfg::kBulkdQ)
-            bwd_dq_tma(smem, bars, tmem_base, &tmAcc, &tmdK, &tmdV, scale, wl, warp - 12, lane);
+            bwd_dq_tma<kStrided>(smem, bars, tmem_base, &tmAcc, &tmdK, &tmdV, scale, wl, warp - 12, lane);
         else
             bwd_dq_tma_wide(smem, bars, tmem_base, &tmAcc, wl, warp - 12, lane);
     }
@@ -864,43 +870,51 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 template <int D, bool kCausal>
 cudaError_t launch_one(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV,
                        const CUtensorMap& tmdO, const CUtensorMap& tmAcc, const CUtensorMap& tmdK,
-                       const CUtensorMap& tmdV, const float* LSE, const float* Delta,
-                       __nv_bfloat16* dK, __nv_bfloat16* dV, const AttnShape& s, int num_sms, int* dev_status,
-                       cudaStream_t stream) {
+                       const CUtensorMap& tmdV, bool strided, uint32_t orders, const float* LSE, const float* Delta,
+                       __nv_bfloat16* dK, __nv_bfloat16* dV, const TensorStrides& sdk, const TensorStrides& sdv,
+                       const AttnShape& s, int num_sms, int* dev_status, cudaStream_t stream) {
     const int n_tiles = (s.T + kBlockK - 1) / kBlockK;
     const int BH = s.B * s.H;
     const long long n_items = static_cast<long long>(n_tiles) * BH;
     const dim3 grid(static_cast<unsigned>(n_items < num_sms ? n_items : num_sms));  // one persistent CTA per SM
-    return launch_overlapped(attn_bwd_kernel<D, kCausal>, grid, dim3(kBwdThreads), BwdCfg<D>::kSmemBytes, stream, tmQ,
-                             tmK, tmV, tmdO, tmAcc, tmdK, tmdV, LSE, Delta, dK, dV, s.T, BH, n_tiles, s.scale,
-                             dev_status);
+    if (strided)
+        return launch_overlapped(attn_bwd_kernel<D, kCausal, true>, grid, dim3(kBwdThreads), BwdCfg<D>::kSmemBytes,
+                                 stream, tmQ, tmK, tmV, tmdO, tmAcc, tmdK, tmdV, LSE, Delta, dK, dV, sdk, sdv, s.T, BH, s.H,
+                                 orders, n_tiles, s.scale, dev_status);
+    return launch_overlapped(attn_bwd_kernel<D, kCausal, false>, grid, dim3(kBwdThreads), BwdCfg<D>::kSmemBytes, stream,
+                             tmQ, tmK, tmV, tmdO, tmAcc, tmdK, tmdV, LSE, Delta, dK, dV, sdk, sdv, s.T, BH, s.H, orders,
+                             n_tiles, s.scale, dev_status);
+}
+
+template <int D, bool kCausal, bool kStrided>
+cudaError_t configure_one() {
+    return cudaFuncSetAttribute(attn_bwd_kernel<D, kCausal, kStrided>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                BwdCfg<D>::kSmemBytes);
 }
 
 }  // namespace
 
 cudaError_t configure_attn_bwd() {
-    cudaError_t e;
-    e = cudaFuncSetAttribute(attn_bwd_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdCfg<64>::kSmemBytes);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(attn_bwd_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdCfg<64>::kSmemBytes);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(attn_bwd_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdCfg<128>::kSmemBytes);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(attn_bwd_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdCfg<128>::kSmemBytes);
-    return e;
+    const cudaError_t r[8] = {configure_one<64, true, false>(),  configure_one<64, false, false>(),
+                              configure_one<128, true, false>(), configure_one<128, false, false>(),
+                              configure_one<64, true, true>(),   configure_one<64, false, true>(),
+                              configure_one<128, true, true>(),  configure_one<128, false, true>()};
+    for (cudaError_t e : r)
+        if (e != cudaSuccess) return e;
+    return cudaSuccess;
 }
 
 cudaError_t launch_attn_bwd(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV,
                             const CUtensorMap& tmdO, const CUtensorMap& tmAcc, const CUtensorMap& tmdK,
-                            const CUtensorMap& tmdV, const float* LSE, const float* Delta,
-                            __nv_bfloat16* dK, __nv_bfloat16* dV, const AttnShape& s, int num_sms, int* dev_status,
-                            cudaStream_t stream) {
+                            const CUtensorMap& tmdV, bool strided, uint32_t orders, const float* LSE, const float* Delta,
+                            __nv_bfloat16* dK, __nv_bfloat16* dV, const TensorStrides& sdk, const TensorStrides& sdv,
+                            const AttnShape& s, int num_sms, int* dev_status, cudaStream_t stream) {
     if (s.D == 64) {
-        return s.causal ? launch_one<64, true>(tmQ, tmK, tmV, tmdO, tmAcc, tmdK, tmdV, LSE, Delta, dK, dV, s, num_sms, dev_status, stream)
-                        : launch_one<64, false>(tmQ, tmK, tmV, tmdO, tmAcc, tmdK, tmdV, LSE, Delta, dK, dV, s, num_sms, dev_status, stream);
+        return s.causal ? launch_one<64, true>(tmQ, tmK, tmV, tmdO, tmAcc, tmdK, tmdV, strided, orders, LSE, Delta, dK, dV, sdk, sdv, s, num_sms, dev_status, stream)
+                        : launch_one<64, false>(tmQ, tmK, tmV, tmdO, tmAcc, tmdK, tmdV, strided, orders, LSE, Delta, dK, dV, sdk, sdv, s, num_sms, dev_status, stream);
     }
-    return s.causal ? launch_one<128, true>(tmQ, tmK, tmV, tmdO, tmAcc, tmdK, tmdV, LSE, Delta, dK, dV, s, num_sms, dev_status, stream)
-                    : launch_one<128, false>(tmQ, tmK, tmV, tmdO, tmAcc, tmdK, tmdV, LSE, Delta, dK, dV, s, num_sms, dev_status, stream);
+    return s.causal ? launch_one<128, true>(tmQ, tmK, tmV, tmdO, tmAcc, tmdK, tmdV, strided, orders, LSE, Delta, dK, dV, sdk, sdv, s, num_sms, dev_status, stream)
+                    : launch_one<128, false>(tmQ, tmK, tmV, tmdO, tmAcc, tmdK, tmdV, strided, orders, LSE, Delta, dK, dV, sdk, sdv, s, num_sms, dev_status, stream);
 }
 
 }  // namespace nova

@@ -3,7 +3,9 @@
 //   dq_convert_kernel:     dQ = bf16(scale * fp32 accumulator)
 //   zero_kernel:           clears the fp32 accumulator before the backward kernel adds into it
 // Both stream their inputs once with 16-byte loads; rows are split over D/8 lanes and reduced with
-// xor-shuffles.  Grids are sized in multiples of the SM count.
+// xor-shuffles.  Grids are sized in multiples of the SM count.  The bf16 tensors may be strided
+// (batch, head and token strides in elements, multiples of 8): a row index r = (b*H + h)*T + t is
+// then split again; the contiguous case skips that arithmetic.
 #include "kernels.h"
 #include "ptx.cuh"
 
@@ -24,10 +26,20 @@ __device__ __forceinline__ float dot8_bf16(const uint4& a, const uint4& b) {
     return acc;
 }
 
+// Offset, in 16-byte units, of row r = (b*H + h)*T + t of a tensor with strides `s`.
+__device__ __forceinline__ long long row_offset16(long long r, int H, int T, const TensorStrides& s) {
+    const long long bh = r / T;
+    const long long t = r - bh * T;
+    const long long b = bh / H;
+    const long long h = bh - b * H;
+    return (b * s.b + h * s.h + t * s.t) >> 3;
+}
+
 // LPR = lanes per row = D/8 (8 for D=64, 16 for D=128); each lane owns 8 consecutive bf16.
-template <int LPR, int UNROLL>
+template <int LPR, int UNROLL, bool kContiguous>
 __global__ void __launch_bounds__(256) bwd_preprocess_kernel(const uint4* __restrict__ O, const uint4* __restrict__ dO,
-                                                             float* __restrict__ Delta, long long rows) {
+                                                             float* __restrict__ Delta, long long rows, int H, int T,
+                                                             const TensorStrides so, const TensorStrides sdo) {
     griddep_launch_dependents();
     griddep_wait();
     const long long tid = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
@@ -41,8 +53,8 @@ __global__ void __launch_bounds__(256) bwd_preprocess_kernel(const uint4* __rest
         for (int u = 0; u < UNROLL; ++u) {
             const long long ru = r + u * rows_per_pass;
             if (ru < rows) {
-                a[u] = __ldg(O + ru * LPR + sub);
-                b[u] = __ldg(dO + ru * LPR + sub);
+                a[u] = __ldg(O + (kContiguous ? ru * LPR : row_offset16(ru, H, T, so)) + sub);
+                b[u] = __ldg(dO + (kContiguous ? ru * LPR : row_offset16(ru, H, T, sdo)) + sub);
             } else {
                 a[u] = make_uint4(0, 0, 0, 0);
                 b[u] = make_uint4(0, 0, 0, 0);
@@ -59,8 +71,10 @@ __global__ void __launch_bounds__(256) bwd_preprocess_kernel(const uint4* __rest
     }
 }
 
+template <bool kContiguous>
 __global__ void __launch_bounds__(256) dq_convert_kernel(const float4* __restrict__ acc, uint4* __restrict__ dQ,
-                                                         long long n8, float scale) {
+                                                         long long n8, float scale, int lpr_shift, int H, int T,
+                                                         const TensorStrides sdq) {
     griddep_launch_dependents();
     griddep_wait();
     const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
@@ -72,7 +86,12 @@ __global__ void __launch_bounds__(256) dq_convert_kernel(const float4* __restric
         v.y = pack_bf16x2(a.z * scale, a.w * scale);
         v.z = pack_bf16x2(b.x * scale, b.y * scale);
         v.w = pack_bf16x2(b.z * scale, b.w * scale);
-        dQ[i] = v;
+        if (kContiguous) {
+            dQ[i] = v;
+        } else {
+            const long long r = i >> lpr_shift;
+            dQ[row_offset16(r, H, T, sdq) + (i - (r << lpr_shift))] = v;
+        }
     }
 }
 
@@ -97,10 +116,18 @@ cudaError_t launch_zero(void* ptr, size_t bytes, int num_sms, cudaStream_t strea
                              static_cast<uint4*>(ptr), n16);
 }
 
+namespace {
+bool is_contiguous(const AttnShape& s, const TensorStrides& st) {
+    return st.t == s.D && st.h == static_cast<long long>(s.T) * s.D && st.b == static_cast<long long>(s.H) * s.T * s.D;
+}
+}  // namespace
+
 cudaError_t launch_attn_bwd_preprocess(const __nv_bfloat16* O, const __nv_bfloat16* dO, float* Delta,
-                                       long long rows, int D, int num_sms, cudaStream_t stream) {
+                                       const AttnShape& s, const TensorStrides& so, const TensorStrides& sdo,
+                                       int num_sms, cudaStream_t stream) {
     constexpr int kThreads = 256, kUnroll = 4;
-    const int lpr = D / 8;
+    const long long rows = static_cast<long long>(s.B) * s.H * s.T;
+    const int lpr = s.D / 8;
     const long long rows_per_block = kThreads / lpr * kUnroll;
     long long blocks = (rows + rows_per_block - 1) / rows_per_block;
     const long long cap = static_cast<long long>(num_sms) * 8;
@@ -109,20 +136,31 @@ cudaError_t launch_attn_bwd_preprocess(const __nv_bfloat16* O, const __nv_bfloat
     const uint4* o4 = reinterpret_cast<const uint4*>(O);
     const uint4* d4 = reinterpret_cast<const uint4*>(dO);
     const dim3 grid(static_cast<unsigned>(blocks));
-    if (D == 64) return launch_overlapped(bwd_preprocess_kernel<8, kUnroll>, grid, dim3(kThreads), 0, stream, o4, d4, Delta, rows);
-    return launch_overlapped(bwd_preprocess_kernel<16, kUnroll>, grid, dim3(kThreads), 0, stream, o4, d4, Delta, rows);
+    const bool contiguous = is_contiguous(s, so) && is_contiguous(s, sdo);
+    auto go = [&](auto kernel) {
+        return launch_overlapped(kernel, grid, dim3(kThreads), 0, stream, o4, d4, Delta, rows, s.H, s.T, so, sdo);
+    };
+    if (s.D == 64) return contiguous ? go(bwd_preprocess_kernel<8, kUnroll, true>) : go(bwd_preprocess_kernel<8, kUnroll, false>);
+    return contiguous ? go(bwd_preprocess_kernel<16, kUnroll, true>) : go(bwd_preprocess_kernel<16, kUnroll, false>);
 }
 
-cudaError_t launch_dq_convert(const float* dq_acc, __nv_bfloat16* dQ, long long n, float scale, int num_sms,
-                              cudaStream_t stream) {
+cudaError_t launch_dq_convert(const float* dq_acc, __nv_bfloat16* dQ, const AttnShape& s, const TensorStrides& sdq,
+                              float scale, int num_sms, cudaStream_t stream) {
     constexpr int kThreads = 256;
-    const long long n8 = n / 8;  // D is a multiple of 8, so n is too
+    const long long n8 = static_cast<long long>(s.B) * s.H * s.T * s.D / 8;  // D is a multiple of 8
     long long blocks = (n8 + kThreads - 1) / kThreads;
     const long long cap = static_cast<long long>(num_sms) * 8;
     if (blocks > cap) blocks = cap;
     if (blocks < 1) blocks = 1;
-    return launch_overlapped(dq_convert_kernel, dim3(static_cast<unsigned>(blocks)), dim3(kThreads), 0, stream,
-                             reinterpret_cast<const float4*>(dq_acc), reinterpret_cast<uint4*>(dQ), n8, scale);
+    const int lpr_shift = (s.D == 64) ? 3 : 4;
+    const dim3 grid(static_cast<unsigned>(blocks));
+    if (is_contiguous(s, sdq))
+        return launch_overlapped(dq_convert_kernel<true>, grid, dim3(kThreads), 0, stream,
+                                 reinterpret_cast<const float4*>(dq_acc), reinterpret_cast<uint4*>(dQ), n8, scale,
+                                 lpr_shift, s.H, s.T, sdq);
+    return launch_overlapped(dq_convert_kernel<false>, grid, dim3(kThreads), 0, stream,
+                             reinterpret_cast<const float4*>(dq_acc), reinterpret_cast<uint4*>(dQ), n8, scale, lpr_shift,
+                             s.H, s.T, sdq);
 }
 
 }  // namespace nova

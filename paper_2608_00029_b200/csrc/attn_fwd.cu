@@ -65,7 +65,8 @@ struct FwdBars {
 
 // This CTA's list of work items: 256-row query blocks, heaviest first, dealt in zig-zag passes.
 struct FwdWork {
-    int n_items, n_ctas, cta, BH, n_blocks, n_kv_all, T;
+    int n_items, n_ctas, cta, BH, n_blocks, n_kv_all, T, H;
+    uint32_t orders;  // coordinate orders of the Q, K, V, O tensor maps, four bits each
     bool causal;
     __device__ __forceinline__ int passes() const { return (n_items + n_ctas - 1) / n_ctas; }
     // Item of pass p: block index, head, and the number of key tiles each query tile visits
@@ -83,7 +84,7 @@ struct FwdWork {
     }
 };
 
-template <int D>
+template <int D, bool kStrided>
 __device__ __forceinline__ void fwd_producer(const CUtensorMap* tmQ, const CUtensorMap* tmK,
                                              const CUtensorMap* tmV, uint8_t* smem, FwdBars* bars,
                                              const FwdWork& wk) {
@@ -95,6 +96,7 @@ __device__ __forceinline__ void fwd_producer(const CUtensorMap* tmQ, const CUten
     for (int p = 0; p < wk.passes() && ok; ++p) {
         int blk, bh, n_a, n_b;
         if (!wk.get(p, &blk, &bh, &n_a, &n_b)) continue;
+        const int head = kStrided ? bh % wk.H : 0, batch = kStrided ? bh / wk.H : 0;
         const int qs = w % Cfg::kQStages;
         const uint32_t qph = (w / Cfg::kQStages) & 1;
         ok = mbar_wait(&bars->q_empty[qs], qph ^ 1, abort_flag);
@@ -105,8 +107,8 @@ __device__ __forceinline__ void fwd_producer(const CUtensorMap* tmQ, const CUten
         for (int t = 0; t < 2; ++t)
 #pragma unroll
             for (int h = 0; h < Cfg::kHalves; ++h)
-                tma_load_3d(smem + Cfg::kOffQ + (qs * 2 + t) * Cfg::kTileBytes + h * kHalfTileBytes, tmQ,
-                            &bars->q_full[qs], h * kBoxCols, blk * kBlockRows + t * kBlockQ, bh);
+                tma_load_tile<kStrided>(smem + Cfg::kOffQ + (qs * 2 + t) * Cfg::kTileBytes + h * kHalfTileBytes, tmQ,
+                              &bars->q_full[qs], wk.orders & 15, h * kBoxCols, blk * kBlockRows + t * kBlockQ, head, batch, bh);
         const int n = max(n_a, n_b);
         for (int j = 0; j < n; ++j, ++g) {
             const int st = g & 1;
@@ -117,16 +119,16 @@ __device__ __forceinline__ void fwd_producer(const CUtensorMap* tmQ, const CUten
             armed_k[st] = ph;
 #pragma unroll
             for (int h = 0; h < Cfg::kHalves; ++h)
-                tma_load_3d(smem + Cfg::kOffK + st * Cfg::kTileBytes + h * kHalfTileBytes, tmK, &bars->k_full[st],
-                            h * kBoxCols, j * kBlockK, bh);
+                tma_load_tile<kStrided>(smem + Cfg::kOffK + st * Cfg::kTileBytes + h * kHalfTileBytes, tmK, &bars->k_full[st],
+                              (wk.orders >> 4) & 15, h * kBoxCols, j * kBlockK, head, batch, bh);
             ok = mbar_wait(&bars->v_empty[st], ph ^ 1, abort_flag);
             if (!ok) break;
             mbar_expect_tx(&bars->v_full[st], Cfg::kTileBytes);
             armed_v[st] = ph;
 #pragma unroll
             for (int h = 0; h < Cfg::kHalves; ++h)
-                tma_load_3d(smem + Cfg::kOffV + st * Cfg::kTileBytes + h * kHalfTileBytes, tmV, &bars->v_full[st],
-                            h * kBoxCols, j * kBlockK, bh);
+                tma_load_tile<kStrided>(smem + Cfg::kOffV + st * Cfg::kTileBytes + h * kHalfTileBytes, tmV, &bars->v_full[st],
+                              (wk.orders >> 8) & 15, h * kBoxCols, j * kBlockK, head, batch, bh);
         }
         ++w;
     }
@@ -278,7 +280,7 @@ __device__ __forceinline__ void fwd_mma(uint8_t* smem, FwdBars* bars, uint32_t t
     }
 }
 
-template <int D, bool kCausal>
+template <int D, bool kCausal, bool kStrided>
 __device__ __forceinline__ void fwd_softmax(uint8_t* smem, FwdBars* bars, uint32_t tmem_base, const CUtensorMap* tmO,
                                             float* __restrict__ LSE, float scale, const FwdWork& wk, int t, int swarp,
                                             int lane) {
@@ -458,7 +460,8 @@ __device__ __forceinline__ void fwd_softmax(uint8_t* smem, FwdBars* bars, uint32
             if (leader_ok) {
 #pragma unroll
                 for (int h = 0; h < Cfg::kHalves; ++h)
-                    tma_store_3d(tmO, stage + h * kHalfTileBytes, h * kBoxCols, qt * kBlockQ, bh);
+                    tma_store_tile<kStrided>(tmO, stage + h * kHalfTileBytes, (wk.orders >> 12) & 15, h * kBoxCols,
+                                             qt * kBlockQ, kStrided ? bh % wk.H : 0, kStrided ? bh / wk.H : 0, bh);
                 bulk_commit_group();
                 bulk_wait_group_read<0>();  // the buffer has been read and may receive the next Q tile
                 mbar_arrive(&bars->q_empty[qs]);
@@ -473,18 +476,19 @@ __device__ __forceinline__ void fwd_softmax(uint8_t* smem, FwdBars* bars, uint32
     if (leader) bulk_wait_group<0>();  // O must be complete before the kernel ends
 }
 
-template <int D, bool kCausal>
+template <int D, bool kCausal, bool kStrided>
 __global__ void __launch_bounds__(kFwdThreads, 1)
 attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
-                float* __restrict__ LSE, int T, int BH, int n_blocks, float scale, int* __restrict__ dev_status) {
+                float* __restrict__ LSE, int T, int BH, int H, uint32_t orders, int n_blocks, float scale,
+                int* __restrict__ dev_status) {
     using Cfg = FwdCfg<D>;
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     FwdBars* bars = reinterpret_cast<FwdBars*>(smem + Cfg::kOffBar);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const FwdWork wk{n_blocks * BH, static_cast<int>(gridDim.x), static_cast<int>(blockIdx.x), BH, n_blocks,
-                     (T + kBlockK - 1) / kBlockK, T, kCausal};
+                     (T + kBlockK - 1) / kBlockK, T, H, orders, kCausal};
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < 2; ++s) {
@@ -521,12 +525,12 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     griddep_wait();  // everything above overlaps the previous kernel of the stream
 
     if (warp == 0) {
-        if (lane == 0) fwd_producer<D>(&tmQ, &tmK, &tmV, smem, bars, wk);
+        if (lane == 0) fwd_producer<D, kStrided>(&tmQ, &tmK, &tmV, smem, bars, wk);
     } else if (warp == 1) {
         fwd_mma<D>(smem, bars, tmem_base, wk);
     } else if (warp >= 4) {
         const int t = (warp - 4) >> 2;
-        fwd_softmax<D, kCausal>(smem, bars, tmem_base, &tmO, LSE, scale, wk, t, (warp - 4) & 3, lane);
+        fwd_softmax<D, kCausal, kStrided>(smem, bars, tmem_base, &tmO, LSE, scale, wk, t, (warp - 4) & 3, lane);
     }
 
     tc_fence_before();
@@ -537,39 +541,46 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 
 template <int D, bool kCausal>
 cudaError_t launch_one(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV,
-                       const CUtensorMap& tmO, float* LSE, const AttnShape& s, int num_sms, int* dev_status,
-                       cudaStream_t stream) {
+                       const CUtensorMap& tmO, bool strided, uint32_t orders, float* LSE, const AttnShape& s,
+                       int num_sms, int* dev_status, cudaStream_t stream) {
     const int n_blocks = (s.T + kBlockRows - 1) / kBlockRows;
     const int BH = s.B * s.H;
     const long long n_items = static_cast<long long>(n_blocks) * BH;
     const dim3 grid(static_cast<unsigned>(n_items < num_sms ? n_items : num_sms));  // one persistent CTA per SM
-    return launch_overlapped(attn_fwd_kernel<D, kCausal>, grid, dim3(kFwdThreads), FwdCfg<D>::kSmemBytes, stream, tmQ,
-                             tmK, tmV, tmO, LSE, s.T, BH, n_blocks, s.scale, dev_status);
+    if (strided)
+        return launch_overlapped(attn_fwd_kernel<D, kCausal, true>, grid, dim3(kFwdThreads), FwdCfg<D>::kSmemBytes,
+                                 stream, tmQ, tmK, tmV, tmO, LSE, s.T, BH, s.H, orders, n_blocks, s.scale, dev_status);
+    return launch_overlapped(attn_fwd_kernel<D, kCausal, false>, grid, dim3(kFwdThreads), FwdCfg<D>::kSmemBytes, stream,
+                             tmQ, tmK, tmV, tmO, LSE, s.T, BH, s.H, orders, n_blocks, s.scale, dev_status);
+}
+
+template <int D, bool kCausal, bool kStrided>
+cudaError_t configure_one() {
+    return cudaFuncSetAttribute(attn_fwd_kernel<D, kCausal, kStrided>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                FwdCfg<D>::kSmemBytes);
 }
 
 }  // namespace
 
 cudaError_t configure_attn_fwd() {
-    cudaError_t e;
-    e = cudaFuncSetAttribute(attn_fwd_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdCfg<64>::kSmemBytes);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(attn_fwd_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdCfg<64>::kSmemBytes);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(attn_fwd_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdCfg<128>::kSmemBytes);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(attn_fwd_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdCfg<128>::kSmemBytes);
-    return e;
+    const cudaError_t r[8] = {configure_one<64, true, false>(),  configure_one<64, false, false>(),
+                              configure_one<128, true, false>(), configure_one<128, false, false>(),
+                              configure_one<64, true, true>(),   configure_one<64, false, true>(),
+                              configure_one<128, true, true>(),  configure_one<128, false, true>()};
+    for (cudaError_t e : r)
+        if (e != cudaSuccess) return e;
+    return cudaSuccess;
 }
 
 cudaError_t launch_attn_fwd(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV,
-                            const CUtensorMap& tmO, float* LSE, const AttnShape& s, int num_sms, int* dev_status,
-                            cudaStream_t stream) {
+                            const CUtensorMap& tmO, bool strided, uint32_t orders, float* LSE, const AttnShape& s,
+                            int num_sms, int* dev_status, cudaStream_t stream) {
     if (s.D == 64) {
-        return s.causal ? launch_one<64, true>(tmQ, tmK, tmV, tmO, LSE, s, num_sms, dev_status, stream)
-                        : launch_one<64, false>(tmQ, tmK, tmV, tmO, LSE, s, num_sms, dev_status, stream);
+        return s.causal ? launch_one<64, true>(tmQ, tmK, tmV, tmO, strided, orders, LSE, s, num_sms, dev_status, stream)
+                        : launch_one<64, false>(tmQ, tmK, tmV, tmO, strided, orders, LSE, s, num_sms, dev_status, stream);
     }
-    return s.causal ? launch_one<128, true>(tmQ, tmK, tmV, tmO, LSE, s, num_sms, dev_status, stream)
-                    : launch_one<128, false>(tmQ, tmK, tmV, tmO, LSE, s, num_sms, dev_status, stream);
+    return s.causal ? launch_one<128, true>(tmQ, tmK, tmV, tmO, strided, orders, LSE, s, num_sms, dev_status, stream)
+                    : launch_one<128, false>(tmQ, tmK, tmV, tmO, strided, orders, LSE, s, num_sms, dev_status, stream);
 }
 
 }  // namespace nova

@@ -19,6 +19,12 @@ struct AttnShape {
     float scale;
 };
 
+// Strides, in elements, of a bf16 tensor indexed [b, h, t, d]; d is contiguous.  [B,H,T,D] storage has
+// (H*T*D, T*D, D); the Q slice of a fused projection output [B, T, 3, H, D] has (T*3*H*D, D, 3*H*D).
+struct TensorStrides {
+    long long b, h, t;
+};
+
 // Launches `kernel` allowing it to overlap the tail of the previous kernel in `stream` (programmatic
 // dependent launch); the kernel must call griddep_wait() before it touches global memory.
 template <typename... KArgs, typename... Args>
@@ -37,15 +43,20 @@ inline cudaError_t launch_overlapped(void (*kernel)(KArgs...), dim3 grid, dim3 b
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
-// Forward: tensor maps are 3-D [D, T, B*H] bf16 with a [64, 128, 1] box and 128-byte swizzle (`tmO`
-// describes the output and is used for TMA stores).  Persistent: launches at most `num_sms` CTAs.
+// Forward.  Two builds of every kernel.  Plain (`strided` false): all bf16 tensors have batch stride =
+// H * head stride, so their maps are 3-D [D, T, B*H]; box of 64 x 128 tokens, 128-byte swizzle.  Strided:
+// the maps are 4-D [D, x, y, z] with token / head / batch in order of increasing stride, and `orders`
+// holds, four bits per tensor in the order Q, K, V, O, which of the three sits where (see
+// tma_load_tile).  `tmO` describes the output and is used for TMA stores.  Persistent: launches at most
+// `num_sms` CTAs.
 cudaError_t launch_attn_fwd(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV,
-                            const CUtensorMap& tmO, float* LSE, const AttnShape& s, int num_sms, int* dev_status,
-                            cudaStream_t stream);
+                            const CUtensorMap& tmO, bool strided, uint32_t orders, float* LSE, const AttnShape& s,
+                            int num_sms, int* dev_status, cudaStream_t stream);
 cudaError_t configure_attn_fwd();
 
 cudaError_t launch_attn_bwd_preprocess(const __nv_bfloat16* O, const __nv_bfloat16* dO, float* Delta,
-                                       long long rows, int D, int num_sms, cudaStream_t stream);
+                                       const AttnShape& s, const TensorStrides& so, const TensorStrides& sdo,
+                                       int num_sms, cudaStream_t stream);
 
 // Exact Delta_i = sum_j P_ij (dO_i . V_j) with P rebuilt from LSE (two contractions + exp2 per tile).
 cudaError_t launch_attn_delta(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV,
@@ -55,20 +66,21 @@ cudaError_t configure_attn_delta();
 
 // Backward main kernel: adds unscaled dQ partial tiles into the fp32 accumulator [B,H,T,D] (zero on
 // entry) described by `tmAcc` (fp32 [D, T, B*H], box [32, 128, 1], 128-byte swizzle) and writes dK and dV
-// (`tmdK`, `tmdV`: the usual bf16 maps of the outputs, used for TMA stores at D=64).
-// Persistent: launches at most `num_sms` CTAs.
+// (`tmdK`, `tmdV`: the bf16 maps of the outputs, used for TMA stores at D=64; at D=128 the rows go out
+// with plain stores through `dK`, `dV` and their strides).  `strided`, `orders`: as in the forward, for
+// Q, K, V, dO, dK, dV.  Persistent: launches at most `num_sms` CTAs.
 cudaError_t launch_attn_bwd(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV,
                             const CUtensorMap& tmdO, const CUtensorMap& tmAcc, const CUtensorMap& tmdK,
-                            const CUtensorMap& tmdV, const float* LSE, const float* Delta,
-                            __nv_bfloat16* dK, __nv_bfloat16* dV, const AttnShape& s, int num_sms, int* dev_status,
-                            cudaStream_t stream);
+                            const CUtensorMap& tmdV, bool strided, uint32_t orders, const float* LSE, const float* Delta,
+                            __nv_bfloat16* dK, __nv_bfloat16* dV, const TensorStrides& sdk, const TensorStrides& sdv,
+                            const AttnShape& s, int num_sms, int* dev_status, cudaStream_t stream);
 cudaError_t configure_attn_bwd();
 
 // Clears `bytes` (a multiple of 16) at the 16-byte aligned `ptr`.
 cudaError_t launch_zero(void* ptr, size_t bytes, int num_sms, cudaStream_t stream);
 
-// dQ = bf16(scale * dq_acc)
-cudaError_t launch_dq_convert(const float* dq_acc, __nv_bfloat16* dQ, long long n, float scale, int num_sms,
-                              cudaStream_t stream);
+// dQ = bf16(scale * dq_acc); the accumulator is contiguous [B,H,T,D], dQ has strides `sdq`.
+cudaError_t launch_dq_convert(const float* dq_acc, __nv_bfloat16* dQ, const AttnShape& s, const TensorStrides& sdq,
+                              float scale, int num_sms, cudaStream_t stream);
 
 }  // namespace nova

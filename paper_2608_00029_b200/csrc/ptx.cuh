@@ -120,6 +120,49 @@ __device__ __forceinline__ void tma_store_3d(const CUtensorMap* m, const void* s
                  "r"(smem_u32(smem_src)), "r"(c0), "r"(c1), "r"(c2)
                  : "memory");
 }
+// Tile copies of the bf16 tensors Q, K, V, O, dO, dK, dV.  The kernels come in two builds.  Plain
+// (kStrided = false): heads and batches merge into one dimension, the maps are 3-D [D, T, B*H] and the
+// coordinate is (d, t, bh).  Strided: the maps are 4-D [D, x, y, z] with token, head and batch in order
+// of increasing stride (so that slices of a fused [B,T,3,H,D] projection output can be read in place);
+// `order` says which of the three sits where: 0: (t,h,b)  1: (h,t,b)  2: (t,b,h)  3: (b,t,h)  4: (h,b,t)
+// 5: (b,h,t).
+__device__ __forceinline__ void tma_order_coords(int order, int t, int h, int b, int& c1, int& c2, int& c3) {
+    switch (order) {
+        case 0: c1 = t; c2 = h; c3 = b; break;
+        case 1: c1 = h; c2 = t; c3 = b; break;
+        case 2: c1 = t; c2 = b; c3 = h; break;
+        case 3: c1 = b; c2 = t; c3 = h; break;
+        case 4: c1 = h; c2 = b; c3 = t; break;
+        default: c1 = b; c2 = h; c3 = t; break;
+    }
+}
+template <bool kStrided>
+__device__ __forceinline__ void tma_load_tile(void* smem_dst, const CUtensorMap* m, uint64_t* bar, int order, int d,
+                                              int t, int h, int b, int bh) {
+    if constexpr (!kStrided) {
+        tma_load_3d(smem_dst, m, bar, d, t, bh);
+        return;
+    }
+    int c1, c2, c3;
+    tma_order_coords(order, t, h, b, c1, c2, c3);
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(smem_u32(smem_dst)), "l"(m), "r"(smem_u32(bar)), "r"(d), "r"(c1), "r"(c2), "r"(c3)
+        : "memory");
+}
+template <bool kStrided>
+__device__ __forceinline__ void tma_store_tile(const CUtensorMap* m, const void* smem_src, int order, int d, int t,
+                                               int h, int b, int bh) {
+    if constexpr (!kStrided) {
+        tma_store_3d(m, smem_src, d, t, bh);
+        return;
+    }
+    int c1, c2, c3;
+    tma_order_coords(order, t, h, b, c1, c2, c3);
+    asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5}], [%1];" ::"l"(m),
+                 "r"(smem_u32(smem_src)), "r"(d), "r"(c1), "r"(c2), "r"(c3)
+                 : "memory");
+}
 // Make generic-proxy writes to shared memory visible to the async proxy (TMA, UMMA operand reads).
 __device__ __forceinline__ void fence_proxy_async_smem() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");

@@ -3,7 +3,10 @@ paper's attention microbenchmark (Section 6, "Attention": sequence lengths 512 t
 heads, head dimension 64 or 128; the figure with the per-shape values is an image, so the eight points
 here are chosen inside those ranges, at batch 16 like the figure's "16x12x64" label).
 
-    python -m paper_2608_00029_b200.grid_case [--batch 16] [--reps 30] [--non-causal]
+    python -m paper_2608_00029_b200.grid_case [--batch 16] [--reps 30] [--non-causal] [--fused]
+
+--fused times the strided entry points on the fused-projection layout instead: Q, K, V read in place from
+a [B, T, 3, H, D] buffer, O and dO as [B, T, H, D], dQ, dK, dV written into a [B, T, 3, H, D] buffer.
 
 Prints one markdown table row per shape: milliseconds and counted TFLOP/s (forward 2*B*H*T^2*D for the
 causal case, backward 2.5x that; twice as much without the mask) of nova_attn_fwd and of
@@ -42,6 +45,7 @@ def main():
     ap.add_argument("--batch", type=int, default=16)
     ap.add_argument("--reps", type=int, default=30)
     ap.add_argument("--non-causal", action="store_true")
+    ap.add_argument("--fused", action="store_true")
     args = ap.parse_args()
     causal = not args.non_causal
     dev = torch.device("cuda:0")
@@ -55,12 +59,31 @@ def main():
         delta = torch.empty_like(lse)
         ws = torch.empty(na.nova_attn_bwd_workspace_bytes(cfg.B, H, T, D), dtype=torch.uint8, device=dev)
 
-        def fwd():
-            na.nova_attn_fwd(q, k, v, o, lse, cfg.scale, causal)
+        if args.fused:
+            B = cfg.B
+            qkv = torch.empty((B, T, 3, H, D), dtype=torch.bfloat16, device=dev)
+            for i, x in enumerate((q, k, v)):
+                qkv[:, :, i] = x.permute(0, 2, 1, 3)
+            dqkv = torch.empty_like(qkv)
+            o_buf = torch.empty((B, T, H, D), dtype=torch.bfloat16, device=dev)
+            do_buf = do.permute(0, 2, 1, 3).contiguous()
+            q, k, v = (qkv[:, :, i].permute(0, 2, 1, 3) for i in range(3))
+            dq, dk, dv = (dqkv[:, :, i].permute(0, 2, 1, 3) for i in range(3))
+            o, do = o_buf.permute(0, 2, 1, 3), do_buf.permute(0, 2, 1, 3)
 
-        def bwd():
-            na.nova_attn_bwd_preprocess(o, do, delta)
-            na.nova_attn_bwd(q, k, v, o, do, lse, delta, dq, dk, dv, cfg.scale, causal, ws)
+            def fwd():
+                na.nova_attn_fwd_strided(q, k, v, o, lse, cfg.scale, causal)
+
+            def bwd():
+                na.nova_attn_bwd_preprocess_strided(o, do, delta)
+                na.nova_attn_bwd_strided(q, k, v, do, lse, delta, dq, dk, dv, cfg.scale, causal, ws)
+        else:
+            def fwd():
+                na.nova_attn_fwd(q, k, v, o, lse, cfg.scale, causal)
+
+            def bwd():
+                na.nova_attn_bwd_preprocess(o, do, delta)
+                na.nova_attn_bwd(q, k, v, o, do, lse, delta, dq, dk, dv, cfg.scale, causal, ws)
 
         t_f, t_b = _time(fwd, args.reps), _time(bwd, args.reps)
         f_flops = cfg.fwd_flops * (1.0 if causal else 2.0)  # the counted figure covers half the square
@@ -68,7 +91,7 @@ def main():
         na.nova_attn_poll_device_status()
         print(f"| {cfg.B} | {H} | {T} | {D} | {'yes' if causal else 'no'} | {t_f:.4f} | {f_flops / t_f / 1e9:.0f} | "
               f"{t_b:.4f} | {b_flops / t_b / 1e9:.0f} | {t_f + t_b:.4f} |", flush=True)
-        del q, k, v, do, o, dq, dk, dv, lse, delta, ws
+        del q, k, v, do, o, dq, dk, dv, lse, delta, ws, fwd, bwd
         torch.cuda.empty_cache()
 
 

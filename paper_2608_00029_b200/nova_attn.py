@@ -19,6 +19,11 @@ OK = 0
 ERR_NULL, ERR_SHAPE, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_SCALE, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(-1, -9, -1)
 
 
+class Strides(ctypes.Structure):
+    """nova_attn_strides: element strides of a tensor addressed (b, h, t, d), d contiguous."""
+    _fields_ = [("batch", ctypes.c_longlong), ("head", ctypes.c_longlong), ("token", ctypes.c_longlong)]
+
+
 class NovaAttnError(RuntimeError):
     def __init__(self, status: int, where: str):
         self.status = status
@@ -51,6 +56,13 @@ def load():
     lib.nova_attn_bwd.restype = i
     lib.nova_attn_bwd_steps.argtypes = [vp] * 5 + [fp, fp, vp, vp, vp, i, i, i, i, f, i, vp, sz, vp, i]
     lib.nova_attn_bwd_steps.restype = i
+    sp = ctypes.POINTER(Strides)
+    lib.nova_attn_fwd_strided.argtypes = [vp, vp, vp, vp, fp, i, i, i, i, sp, sp, sp, sp, f, i, vp]
+    lib.nova_attn_fwd_strided.restype = i
+    lib.nova_attn_bwd_preprocess_strided.argtypes = [vp, vp, fp, i, i, i, i, sp, sp, vp]
+    lib.nova_attn_bwd_preprocess_strided.restype = i
+    lib.nova_attn_bwd_strided.argtypes = [vp] * 4 + [fp, fp, vp, vp, vp, i, i, i, i] + [sp] * 7 + [f, i, vp, sz, vp]
+    lib.nova_attn_bwd_strided.restype = i
     lib.nova_attn_status_string.argtypes = [i]
     lib.nova_attn_status_string.restype = ctypes.c_char_p
     lib.nova_attn_last_cuda_error.argtypes = []
@@ -80,6 +92,16 @@ def _check_bf16(name, t, shape=None):
         raise TypeError(f"{name} must be a contiguous CUDA bf16 tensor")
     if shape is not None and tuple(t.shape) != tuple(shape):
         raise ValueError(f"{name} has shape {tuple(t.shape)}, expected {tuple(shape)}")
+
+
+def _view_strides(name, t, shape=None) -> Strides:
+    """Strides of a [B,H,T,D]-shaped bf16 CUDA view whose last dimension is contiguous (the view may be a
+    slice / permutation of a larger buffer, e.g. of a fused projection output)."""
+    if t.dtype != torch.bfloat16 or not t.is_cuda or t.dim() != 4 or t.stride(3) != 1:
+        raise TypeError(f"{name} must be a 4-D CUDA bf16 view [B,H,T,D] with a contiguous last dimension")
+    if shape is not None and tuple(t.shape) != tuple(shape):
+        raise ValueError(f"{name} has shape {tuple(t.shape)}, expected {tuple(shape)}")
+    return Strides(t.stride(0), t.stride(1), t.stride(2))
 
 
 def _check_f32(name, t, shape):
@@ -191,3 +213,47 @@ def nova_attn_poll_device_status(stream=None) -> int:
     if rc != OK:
         raise NovaAttnError(rc, "nova_attn_poll_device_status")
     return rc
+
+
+def nova_attn_fwd_strided(Q, K, V, O, LSE, scale: float, causal: bool = True, stream=None) -> None:
+    """nova_attn_fwd on [B,H,T,D]-shaped VIEWS: strides are taken from the tensors, so Q, K, V may be slices
+    of a fused projection output and O a permuted view of a [B,T,H,D] buffer.  LSE is contiguous [B,H,T]."""
+    sq = _view_strides("Q", Q)
+    B, H, T, D = Q.shape
+    sk, sv, so = (_view_strides(n, t, Q.shape) for n, t in (("K", K), ("V", V), ("O", O)))
+    _check_f32("LSE", LSE, (B, H, T))
+    rc = load().nova_attn_fwd_strided(_ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(LSE), B, H, T, D, sq, sk, sv, so,
+                                      float(scale), int(bool(causal)), _stream_ptr(stream))
+    if rc != OK:
+        raise NovaAttnError(rc, "nova_attn_fwd_strided")
+
+
+def nova_attn_bwd_preprocess_strided(O, dO, Delta, stream=None) -> None:
+    """nova_attn_bwd_preprocess on [B,H,T,D]-shaped views."""
+    so = _view_strides("O", O)
+    sdo = _view_strides("dO", dO, O.shape)
+    B, H, T, D = O.shape
+    _check_f32("Delta", Delta, (B, H, T))
+    rc = load().nova_attn_bwd_preprocess_strided(_ptr(O), _ptr(dO), _ptr(Delta), B, H, T, D, so, sdo,
+                                                 _stream_ptr(stream))
+    if rc != OK:
+        raise NovaAttnError(rc, "nova_attn_bwd_preprocess_strided")
+
+
+def nova_attn_bwd_strided(Q, K, V, dO, LSE, Delta, dQ, dK, dV, scale: float, causal: bool = True, workspace=None,
+                          stream=None) -> None:
+    """nova_attn_bwd on [B,H,T,D]-shaped views (dQ, dK, dV may be slices of one fused gradient buffer)."""
+    sq = _view_strides("Q", Q)
+    B, H, T, D = Q.shape
+    rest = [_view_strides(n, t, Q.shape) for n, t in (("K", K), ("V", V), ("dO", dO), ("dQ", dQ), ("dK", dK), ("dV", dV))]
+    _check_f32("LSE", LSE, (B, H, T))
+    _check_f32("Delta", Delta, (B, H, T))
+    need = nova_attn_bwd_workspace_bytes(B, H, T, D)
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=Q.device)
+    rc = load().nova_attn_bwd_strided(_ptr(Q), _ptr(K), _ptr(V), _ptr(dO), _ptr(LSE), _ptr(Delta), _ptr(dQ), _ptr(dK),
+                                      _ptr(dV), B, H, T, D, sq, *rest, float(scale), int(bool(causal)),
+                                      _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                      _stream_ptr(stream))
+    if rc != OK:
+        raise NovaAttnError(rc, "nova_attn_bwd_strided")

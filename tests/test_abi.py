@@ -76,6 +76,30 @@ def test_host_side_validation_rejects_before_launch(lib):
     assert e(p, p, p, p, p, p, 1, 1, 16, 64, -2.0, 1, None) == na.ERR_SCALE
 
 
+def test_strided_entry_points_validate_strides(lib):
+    from paper_2608_00029_b200 import nova_attn as na
+    p = ctypes.c_void_p(0x1000)
+    S = na.Strides
+    good = S(16 * 3 * 2 * 64, 64, 3 * 2 * 64)            # the Q slice of a fused [B, T, 3, H=2, D=64] buffer
+    f = lib.nova_attn_fwd_strided
+    base = (p, p, p, p, p, 1, 2, 16, 64)
+    assert f(*base, None, good, good, good, 1.0, 1, None) == na.ERR_NULL
+    assert f(*base, good, S(100, 64, 384), good, good, 1.0, 1, None) == na.ERR_ALIGNMENT   # 100 % 8 != 0
+    assert f(*base, good, good, S(6144, 64, 32), good, 1.0, 1, None) == na.ERR_SHAPE        # token stride < D
+    assert f(*base, good, good, good, S(6144, 0, 384), 1.0, 1, None) == na.ERR_SHAPE
+    assert f(*base, good, good, good, S(1 << 40, 64, 384), 1.0, 1, None) == na.ERR_SHAPE
+    assert f(*base, good, good, good, good, 0.0, 1, None) == na.ERR_SCALE
+    g = lib.nova_attn_bwd_preprocess_strided
+    assert g(p, p, p, 1, 2, 16, 64, good, None, None) == na.ERR_NULL
+    assert g(p, p, p, 1, 2, 16, 64, good, S(6144, 64, 380), None) == na.ERR_ALIGNMENT
+    b = lib.nova_attn_bwd_strided
+    ptrs = [p] * 9
+    seven = [good] * 7
+    assert b(*ptrs, 1, 2, 16, 64, *seven, 1.0, 1, None, 0, None) == na.ERR_WORKSPACE
+    seven[4] = S(6144, 64, 8)
+    assert b(*ptrs, 1, 2, 16, 64, *seven, 1.0, 1, p, 1 << 20, None) == na.ERR_SHAPE
+
+
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     from paper_2608_00029_b200 import nova_attn as na
     monkeypatch.setattr(na, "_lib", None)

@@ -257,3 +257,53 @@ def test_back_to_back_steps_on_shared_buffers():
         assert torch.equal(dk_s.cpu(), r["dK"]) and torch.equal(dv_s.cpu(), r["dV"])
         d = (dq_s.cpu().float() - r["dQ"].float()).abs().max()
         assert d <= 1e-2 * r["dQ"].float().abs().max()  # dQ: summation order of the reduce-adds
+
+
+FUSED = [  # (B, H, T, D, causal)
+    (2, 3, 300, 64, True),      # ragged T: partial tiles with TMA clipping on strided rows
+    (2, 12, 1024, 64, True),    # the GPT-2 layout: H*D = 768
+    (1, 4, 384, 128, True),     # D = 128: dK/dV rows leave through plain strided stores
+    (2, 2, 256, 64, False),
+]
+
+
+@pytest.mark.parametrize("B,H,T,D,causal", FUSED)
+def test_fused_projection_layout(B, H, T, D, causal):
+    """Q, K, V read straight out of a fused projection output [B, T, 3, H, D]; O written as [B, T, H, D]; dO
+    given as [B, T, H, D]; dQ, dK, dV written into one fused gradient buffer [B, T, 3, H, D] (paper
+    Section 4.2: the per-head layout change costs nothing).  Only the addressing differs from the
+    [B,H,T,D] entry points, so O, LSE, Delta, dK, dV must be bit-identical to theirs; and both match the oracle."""
+    from paper_2608_00029_b200 import nova_attn
+    h = _harness()
+    dev = torch.device("cuda:0")
+    cfg = W.AttnConfig("fused", B=B, H=H, T=T, D=D, seed=500 + T + D, causal=causal)
+    Q, K, V, dO = W.make_inputs(cfg)
+    plain = h.run_gpu(Q, K, V, dO, cfg.scale, causal)
+
+    qkv = torch.full((B, T, 3, H, D), 7.0, dtype=torch.bfloat16, device=dev)
+    for i, x in enumerate((Q, K, V)):
+        qkv[:, :, i] = x.to(dev).permute(0, 2, 1, 3)
+    q_v, k_v, v_v = (qkv[:, :, i].permute(0, 2, 1, 3) for i in range(3))        # [B,H,T,D] views, no copy
+    assert q_v.data_ptr() == qkv.data_ptr() and k_v.data_ptr() == qkv.data_ptr() + 2 * H * D
+    o_buf = torch.full((B, T, H, D), 7.0, dtype=torch.bfloat16, device=dev)
+    do_buf = dO.to(dev).permute(0, 2, 1, 3).contiguous()                        # [B,T,H,D]
+    dqkv = torch.full((B, T, 3, H, D), 7.0, dtype=torch.bfloat16, device=dev)
+    o_v, do_v = o_buf.permute(0, 2, 1, 3), do_buf.permute(0, 2, 1, 3)
+    dq_v, dk_v, dv_v = (dqkv[:, :, i].permute(0, 2, 1, 3) for i in range(3))
+    lse = torch.empty((B, H, T), dtype=torch.float32, device=dev)
+    delta = torch.empty_like(lse)
+    nova_attn.nova_attn_fwd_strided(q_v, k_v, v_v, o_v, lse, cfg.scale, causal)
+    nova_attn.nova_attn_bwd_preprocess_strided(o_v, do_v, delta)
+    nova_attn.nova_attn_bwd_strided(q_v, k_v, v_v, do_v, lse, delta, dq_v, dk_v, dv_v, cfg.scale, causal)
+    nova_attn.nova_attn_poll_device_status()
+    assert torch.equal(qkv[:, :, 0].permute(0, 2, 1, 3).cpu(), Q), "inputs must not be modified"
+
+    got = {"O": o_v.contiguous().cpu(), "LSE": lse.cpu(), "Delta": delta.cpu(),
+           "dQ": dq_v.contiguous().cpu(), "dK": dk_v.contiguous().cpu(), "dV": dv_v.contiguous().cpu()}
+    for name in ("O", "LSE", "Delta", "dK", "dV"):
+        assert torch.equal(got[name], plain[name]), f"{name}: strided and contiguous entry points differ"
+    d = (got["dQ"].float() - plain["dQ"].float()).abs().max()
+    assert d <= 1e-2 * plain["dQ"].float().abs().max()
+    heads = sorted({(i % B, (i * 5 + 1) % H) for i in range(4)})
+    ref = h.run_oracle(Q, K, V, dO, cfg.scale, causal, heads=heads)
+    h.compare(h.select_heads(got, heads), ref, label=f"fused T={T} D={D}: ", dO=ref["dO_in"])
