@@ -162,6 +162,23 @@ int nova_attn_bwd_static_scratch(const void* Q, const void* K, const void* V, co
                                  float scale, int causal, void* stream);
 
 /*
+ * Deterministic backward: the two-kernel form of the paper (Section 4.2, "The Backward Pass": one kernel
+ * reduces dQ over keys, the other reduces dK and dV over queries; both rebuild the probability matrix from
+ * the saved log-sum-exp).  Every output element is summed by one thread block in a fixed order, so dQ, dK
+ * and dV are bitwise reproducible from run to run, and no workspace is needed.  The price: the score and
+ * dP contractions are computed in both kernels (seven contractions for the five that are counted) and
+ * the dQ kernel keeps one query tile in flight per SM, so it is slower than nova_attn_bwd; dK and dV are
+ * bit-identical to nova_attn_bwd's, dQ differs from it in the last bits only (summation order).
+ *   Q, K, V, dO : in,  bf16 [B,H,T,D]
+ *   LSE, Delta  : in,  fp32 [B,H,T] from nova_attn_fwd / nova_attn_bwd_preprocess(_exact)
+ *   dQ, dK, dV  : out, bf16 [B,H,T,D]
+ * Validation and errors as for nova_attn_bwd (without the workspace).
+ */
+int nova_attn_bwd_deterministic(const void* Q, const void* K, const void* V, const void* dO,
+                                const float* LSE, const float* Delta, void* dQ, void* dK, void* dV,
+                                int B, int H, int T, int D, float scale, int causal, void* stream);
+
+/*
  * Strided variants (paper Section 4.2: the per-head layout change around attention is expressed in the
  * access pattern, so the transposes between the fused projection output and the per-head tensors cost
  * nothing).  Each bf16 tensor is addressed as element (b, h, t, d) at

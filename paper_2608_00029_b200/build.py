@@ -8,7 +8,8 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libnova_attn.so")
-SOURCES = ["api.cu", "attn_fwd.cu", "attn_bwd.cu", "attn_bwd_pre.cu", "attn_delta.cu", "attn_bwd_static.cu"]
+SOURCES = ["api.cu", "attn_fwd.cu", "attn_bwd.cu", "attn_bwd_pre.cu", "attn_delta.cu", "attn_dq.cu",
+           "attn_bwd_static.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-shared", "-cudart", "shared"]
 

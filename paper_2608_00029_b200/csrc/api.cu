@@ -70,6 +70,7 @@ int device_state(DeviceState** out) {
         e = configure_attn_fwd();
         if (e == cudaSuccess) e = configure_attn_bwd();
         if (e == cudaSuccess) e = configure_attn_delta();
+        if (e == cudaSuccess) e = configure_attn_dq();
         if (e == cudaSuccess) e = cudaGetSymbolAddress(reinterpret_cast<void**>(&st.dev_status), g_dev_status);
         if (e != cudaSuccess) { st.status = fail_cuda(e); return st.status; }
     }
@@ -376,7 +377,7 @@ int bwd_impl(const void* Q, const void* K, const void* V, const void* dO, const 
         if (int rc = get_bf16_map(dK, s, sdk, strided, &tmdK, &odk)) return rc;
         if (int rc = get_bf16_map(dV, s, sdv, strided, &tmdV, &odv)) return rc;
         const uint32_t orders = oq | (ok << 4) | (ov << 8) | (odo << 12) | (odk << 16) | (odv << 20);
-        e = launch_attn_bwd(tmQ, tmK, tmV, tmdO, tmAcc, tmdK, tmdV, strided, orders, LSE, Delta, static_cast<__nv_bfloat16*>(dK),
+        e = launch_attn_bwd(tmQ, tmK, tmV, tmdO, tmAcc, tmdK, tmdV, strided, orders, false, LSE, Delta, static_cast<__nv_bfloat16*>(dK),
                             static_cast<__nv_bfloat16*>(dV), sdk, sdv, s, st->num_sms, st->dev_status, cs);
         if (e != cudaSuccess) return fail_cuda(e);
     }
@@ -404,6 +405,36 @@ int nova_attn_bwd(const void* Q, const void* K, const void* V, const void* O, co
     return nova_attn_bwd_steps(Q, K, V, O, dO, LSE, Delta, dQ, dK, dV, B, H, T, D, scale, causal, workspace,
                                workspace_bytes, stream,
                                NOVA_ATTN_BWD_STEP_ZERO | NOVA_ATTN_BWD_STEP_MAIN | NOVA_ATTN_BWD_STEP_CONVERT);
+}
+
+int nova_attn_bwd_deterministic(const void* Q, const void* K, const void* V, const void* dO, const float* LSE,
+                                const float* Delta, void* dQ, void* dK, void* dV, int B, int H, int T, int D,
+                                float scale, int causal, void* stream) {
+    if (!Q || !K || !V || !dO || !LSE || !Delta || !dQ || !dK || !dV) return NOVA_ATTN_ERR_NULL;
+    if (int rc = check_shape(B, H, T, D)) return rc;
+    if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(dO) || !aligned16(LSE) || !aligned16(Delta) ||
+        !aligned16(dQ) || !aligned16(dK) || !aligned16(dV))
+        return NOVA_ATTN_ERR_ALIGNMENT;
+    if (!std::isfinite(scale) || !(scale > 0.f)) return NOVA_ATTN_ERR_SCALE;
+    DeviceState* st = nullptr;
+    if (int rc = device_state(&st)) return rc;
+    const long long BH = static_cast<long long>(B) * H;
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    const AttnShape s{B, H, T, D, causal != 0, scale};
+    const TensorStrides c = contiguous_strides(H, T, D);
+    CUtensorMap tmQ, tmK, tmV, tmdO, tmdK, tmdV;
+    if (int rc = get_tensor_map(Q, D, T, BH, &tmQ)) return rc;
+    if (int rc = get_tensor_map(K, D, T, BH, &tmK)) return rc;
+    if (int rc = get_tensor_map(V, D, T, BH, &tmV)) return rc;
+    if (int rc = get_tensor_map(dO, D, T, BH, &tmdO)) return rc;
+    if (int rc = get_tensor_map(dK, D, T, BH, &tmdK)) return rc;
+    if (int rc = get_tensor_map(dV, D, T, BH, &tmdV)) return rc;
+    cudaError_t e = launch_attn_dq(tmQ, tmK, tmV, tmdO, LSE, Delta, static_cast<__nv_bfloat16*>(dQ), s, st->dev_status, cs);
+    if (e != cudaSuccess) return fail_cuda(e);
+    // the dK/dV half: the fused kernel without its dQ product (the accumulator map is never used: any map will do)
+    e = launch_attn_bwd(tmQ, tmK, tmV, tmdO, tmQ, tmdK, tmdV, false, 0u, true, LSE, Delta, static_cast<__nv_bfloat16*>(dK),
+                        static_cast<__nv_bfloat16*>(dV), c, c, s, st->num_sms, st->dev_status, cs);
+    return e == cudaSuccess ? NOVA_ATTN_OK : fail_cuda(e);
 }
 
 int nova_attn_bwd_strided(const void* Q, const void* K, const void* V, const void* dO, const float* LSE,

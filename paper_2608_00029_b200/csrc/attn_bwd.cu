@@ -105,6 +105,7 @@ struct BwdBars {
 struct WorkList {
     int n_items, n_ctas, cta, BH, n_tiles, H;
     uint32_t orders;  // coordinate orders of the Q, K, V, dO, dK, dV tensor maps, four bits each
+    bool no_dq;       // dK/dV half of the two-kernel backward: no dQ product, no accumulator traffic
     bool causal;
     __device__ __forceinline__ int passes() const { return (n_items + n_ctas - 1) / n_ctas; }
     // Item of pass p: returns false if this CTA has none in that pass.
@@ -252,7 +253,7 @@ __device__ __forceinline__ void bwd_mma(uint8_t* smem, BwdBars* bars, uint32_t t
         v_k = umma_desc_lo(smem_u32(smem + Cfg::kOffV + ks * Cfg::kTileBytes), 16);
         ok = mbar_wait(&bars->kv_full[ks], (w / Cfg::kKVStages) & 1, abort_flag);
         if (ok) ok = mbar_wait(&bars->q_full[g & 1], (g >> 1) & 1, abort_flag);
-        if (ok && Cfg::kdQAliased && g > 0) ok = mbar_wait(&bars->dq_free, (g - 1) & 1, abort_flag);
+        if (ok && Cfg::kdQAliased && g > 0 && !wl.no_dq) ok = mbar_wait(&bars->dq_free, (g - 1) & 1, abort_flag);
         if (ok) ok = mbar_wait(&bars->do_full[g % Cfg::kdOStages], (g / Cfg::kdOStages) & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
@@ -311,12 +312,12 @@ __device__ __forceinline__ void bwd_mma(uint8_t* smem, BwdBars* bars, uint32_t t
             }
             __syncwarp();
             // dQ_i = dS K_j, 64 head-dim columns per accumulator half; 16 keys per instruction.
-            if (!Cfg::kdQAliased) {  // the dQ warps must have read the previous tile out of the dQ columns
+            if (!Cfg::kdQAliased && !wl.no_dq) {  // the dQ warps must have read the previous tile out of the dQ columns
                 ok = mbar_wait(&bars->dq_free, (g & 1) ^ 1, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
             }
-            if (el) {
+            if (el && !wl.no_dq) {
 #pragma unroll
                 for (int h = 0; h < Cfg::kHalves; ++h) {
                     const uint32_t t_dq = tmem_base + Cfg::kColdQ + h * 64;
@@ -330,7 +331,7 @@ __device__ __forceinline__ void bwd_mma(uint8_t* smem, BwdBars* bars, uint32_t t
             }
             __syncwarp();
             if (more || cross) {
-                if (Cfg::kdQAliased) {  // dQ sits in the dP^T region until the dQ warps have read it
+                if (Cfg::kdQAliased && !wl.no_dq) {  // dQ sits in the dP^T region until the dQ warps have read it
                     ok = mbar_wait(&bars->dq_free, g & 1, abort_flag);
                     if (!ok) break;
                 }
@@ -528,10 +529,12 @@ __device__ __forceinline__ void bwd_compute(uint8_t* smem, BwdBars* bars, uint32
             }
             tmem_st_x32(t_dp, dd);
             // dS^T row r, this half's 64 queries: eight 16-byte chunks of one 128-byte swizzled row.
+            if (!wl.no_dq) {
 #pragma unroll
-            for (int ch = 0; ch < 8; ++ch)
-                *reinterpret_cast<uint4*>(sdS_row + ((ch ^ (r & 7)) << 4)) =
-                    make_uint4(dd[ch * 4 + 0], dd[ch * 4 + 1], dd[ch * 4 + 2], dd[ch * 4 + 3]);
+                for (int ch = 0; ch < 8; ++ch)
+                    *reinterpret_cast<uint4*>(sdS_row + ((ch ^ (r & 7)) << 4)) =
+                        make_uint4(dd[ch * 4 + 0], dd[ch * 4 + 1], dd[ch * 4 + 2], dd[ch * 4 + 3]);
+            }
             tmem_wait_st();
             fence_proxy_async_smem();
             tc_fence_before();
@@ -639,7 +642,7 @@ __device__ __forceinline__ void bwd_dq_tma(uint8_t* smem, BwdBars* bars, uint32_
     for (int p = 0; p < wl.passes() && ok; ++p) {
         int kt, bh, i0, n_it;
         if (!wl.get(p, &kt, &bh, &i0, &n_it)) continue;
-        for (int it = 0; it < n_it; ++it, ++g) {
+        for (int it = 0; it < n_it && !wl.no_dq; ++it, ++g) {
             ok = mbar_wait(&bars->dq_full, g & 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
@@ -753,7 +756,7 @@ __device__ __forceinline__ void bwd_dq_tma_wide(uint8_t* smem, BwdBars* bars, ui
         return __all_sync(0xffffffffu, leader_ok);
     };
 
-    for (int p = 0; p < wl.passes() && ok; ++p) {
+    for (int p = 0; p < wl.passes() && ok && !wl.no_dq; ++p) {
         int kt, bh, i0, n_it;
         if (!wl.get(p, &kt, &bh, &i0, &n_it)) continue;
         for (int it = 0; it < n_it && ok; ++it, ++g) {
@@ -790,7 +793,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 const __grid_constant__ CUtensorMap tmdV, const float* __restrict__ LSE,
                 const float* __restrict__ Delta, __nv_bfloat16* __restrict__ dK,
                 __nv_bfloat16* __restrict__ dV, const TensorStrides sdk, const TensorStrides sdv, int T, int BH,
-                int H, uint32_t orders, int n_tiles, float scale, int* __restrict__ dev_status) {
+                int H, uint32_t orders, int no_dq, int n_tiles, float scale, int* __restrict__ dev_status) {
     using Cfg = BwdCfg<D>;
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -801,7 +804,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     BwdBars* bars = reinterpret_cast<BwdBars*>(smem + Cfg::kOffBar);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const WorkList wl{n_tiles * BH, static_cast<int>(gridDim.x), static_cast<int>(blockIdx.x), BH, n_tiles, H, orders,
-                      kCausal};
+                      no_dq != 0, kCausal};
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < 2; ++s) {
@@ -870,9 +873,9 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 template <int D, bool kCausal>
 cudaError_t launch_one(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV,
                        const CUtensorMap& tmdO, const CUtensorMap& tmAcc, const CUtensorMap& tmdK,
-                       const CUtensorMap& tmdV, bool strided, uint32_t orders, const float* LSE, const float* Delta,
-                       __nv_bfloat16* dK, __nv_bfloat16* dV, const TensorStrides& sdk, const TensorStrides& sdv,
-                       const AttnShape& s, int num_sms, int* dev_status, cudaStream_t stream) {
+                       const CUtensorMap& tmdV, bool strided, uint32_t orders, bool no_dq, const float* LSE,
+                       const float* Delta, __nv_bfloat16* dK, __nv_bfloat16* dV, const TensorStrides& sdk,
+                       const TensorStrides& sdv, const AttnShape& s, int num_sms, int* dev_status, cudaStream_t stream) {
     const int n_tiles = (s.T + kBlockK - 1) / kBlockK;
     const int BH = s.B * s.H;
     const long long n_items = static_cast<long long>(n_tiles) * BH;
@@ -880,10 +883,10 @@ cudaError_t launch_one(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUt
     if (strided)
         return launch_overlapped(attn_bwd_kernel<D, kCausal, true>, grid, dim3(kBwdThreads), BwdCfg<D>::kSmemBytes,
                                  stream, tmQ, tmK, tmV, tmdO, tmAcc, tmdK, tmdV, LSE, Delta, dK, dV, sdk, sdv, s.T, BH, s.H,
-                                 orders, n_tiles, s.scale, dev_status);
+                                 orders, no_dq ? 1 : 0, n_tiles, s.scale, dev_status);
     return launch_overlapped(attn_bwd_kernel<D, kCausal, false>, grid, dim3(kBwdThreads), BwdCfg<D>::kSmemBytes, stream,
                              tmQ, tmK, tmV, tmdO, tmAcc, tmdK, tmdV, LSE, Delta, dK, dV, sdk, sdv, s.T, BH, s.H, orders,
-                             n_tiles, s.scale, dev_status);
+                             no_dq ? 1 : 0, n_tiles, s.scale, dev_status);
 }
 
 template <int D, bool kCausal, bool kStrided>
@@ -906,15 +909,16 @@ cudaError_t configure_attn_bwd() {
 
 cudaError_t launch_attn_bwd(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV,
                             const CUtensorMap& tmdO, const CUtensorMap& tmAcc, const CUtensorMap& tmdK,
-                            const CUtensorMap& tmdV, bool strided, uint32_t orders, const float* LSE, const float* Delta,
-                            __nv_bfloat16* dK, __nv_bfloat16* dV, const TensorStrides& sdk, const TensorStrides& sdv,
-                            const AttnShape& s, int num_sms, int* dev_status, cudaStream_t stream) {
+                            const CUtensorMap& tmdV, bool strided, uint32_t orders, bool no_dq, const float* LSE,
+                            const float* Delta, __nv_bfloat16* dK, __nv_bfloat16* dV, const TensorStrides& sdk,
+                            const TensorStrides& sdv, const AttnShape& s, int num_sms, int* dev_status,
+                            cudaStream_t stream) {
     if (s.D == 64) {
-        return s.causal ? launch_one<64, true>(tmQ, tmK, tmV, tmdO, tmAcc, tmdK, tmdV, strided, orders, LSE, Delta, dK, dV, sdk, sdv, s, num_sms, dev_status, stream)
-                        : launch_one<64, false>(tmQ, tmK, tmV, tmdO, tmAcc, tmdK, tmdV, strided, orders, LSE, Delta, dK, dV, sdk, sdv, s, num_sms, dev_status, stream);
+        return s.causal ? launch_one<64, true>(tmQ, tmK, tmV, tmdO, tmAcc, tmdK, tmdV, strided, orders, no_dq, LSE, Delta, dK, dV, sdk, sdv, s, num_sms, dev_status, stream)
+                        : launch_one<64, false>(tmQ, tmK, tmV, tmdO, tmAcc, tmdK, tmdV, strided, orders, no_dq, LSE, Delta, dK, dV, sdk, sdv, s, num_sms, dev_status, stream);
     }
-    return s.causal ? launch_one<128, true>(tmQ, tmK, tmV, tmdO, tmAcc, tmdK, tmdV, strided, orders, LSE, Delta, dK, dV, sdk, sdv, s, num_sms, dev_status, stream)
-                    : launch_one<128, false>(tmQ, tmK, tmV, tmdO, tmAcc, tmdK, tmdV, strided, orders, LSE, Delta, dK, dV, sdk, sdv, s, num_sms, dev_status, stream);
+    return s.causal ? launch_one<128, true>(tmQ, tmK, tmV, tmdO, tmAcc, tmdK, tmdV, strided, orders, no_dq, LSE, Delta, dK, dV, sdk, sdv, s, num_sms, dev_status, stream)
+                    : launch_one<128, false>(tmQ, tmK, tmV, tmdO, tmAcc, tmdK, tmdV, strided, orders, no_dq, LSE, Delta, dK, dV, sdk, sdv, s, num_sms, dev_status, stream);
 }
 
 }  // namespace nova

@@ -64,14 +64,22 @@ cudaError_t launch_attn_delta(const CUtensorMap& tmQ, const CUtensorMap& tmK, co
                               int* dev_status, cudaStream_t stream);
 cudaError_t configure_attn_delta();
 
+// Deterministic dQ (the dQ half of the paper's two-kernel backward): one CTA per 128-row query tile walks
+// the key tiles in order and writes dQ = bf16(scale * sum_j dS_j K_j).  3-D [D, T, B*H] maps; dQ contiguous.
+cudaError_t launch_attn_dq(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV,
+                           const CUtensorMap& tmdO, const float* LSE, const float* Delta, __nv_bfloat16* dQ,
+                           const AttnShape& s, int* dev_status, cudaStream_t stream);
+cudaError_t configure_attn_dq();
+
 // Backward main kernel: adds unscaled dQ partial tiles into the fp32 accumulator [B,H,T,D] (zero on
 // entry) described by `tmAcc` (fp32 [D, T, B*H], box [32, 128, 1], 128-byte swizzle) and writes dK and dV
 // (`tmdK`, `tmdV`: the bf16 maps of the outputs, used for TMA stores at D=64; at D=128 the rows go out
 // with plain stores through `dK`, `dV` and their strides).  `strided`, `orders`: as in the forward, for
-// Q, K, V, dO, dK, dV.  Persistent: launches at most `num_sms` CTAs.
+// Q, K, V, dO, dK, dV.  `no_dq`: write dK and dV only (the dK/dV half of the two-kernel backward); `tmAcc` is
+// then never used.  Persistent: launches at most `num_sms` CTAs.
 cudaError_t launch_attn_bwd(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV,
                             const CUtensorMap& tmdO, const CUtensorMap& tmAcc, const CUtensorMap& tmdK,
-                            const CUtensorMap& tmdV, bool strided, uint32_t orders, const float* LSE, const float* Delta,
+                            const CUtensorMap& tmdV, bool strided, uint32_t orders, bool no_dq, const float* LSE, const float* Delta,
                             __nv_bfloat16* dK, __nv_bfloat16* dV, const TensorStrides& sdk, const TensorStrides& sdv,
                             const AttnShape& s, int num_sms, int* dev_status, cudaStream_t stream);
 cudaError_t configure_attn_bwd();

@@ -3,7 +3,9 @@ paper's attention microbenchmark (Section 6, "Attention": sequence lengths 512 t
 heads, head dimension 64 or 128; the figure with the per-shape values is an image, so the eight points
 here are chosen inside those ranges, at batch 16 like the figure's "16x12x64" label).
 
-    python -m paper_2608_00029_b200.grid_case [--batch 16] [--reps 30] [--non-causal] [--fused]
+    python -m paper_2608_00029_b200.grid_case [--batch 16] [--reps 30] [--non-causal] [--fused | --deterministic]
+
+--deterministic times nova_attn_bwd_deterministic (the paper's two-kernel backward) as the backward.
 
 --fused times the strided entry points on the fused-projection layout instead: Q, K, V read in place from
 a [B, T, 3, H, D] buffer, O and dO as [B, T, H, D], dQ, dK, dV written into a [B, T, 3, H, D] buffer.
@@ -46,6 +48,7 @@ def main():
     ap.add_argument("--reps", type=int, default=30)
     ap.add_argument("--non-causal", action="store_true")
     ap.add_argument("--fused", action="store_true")
+    ap.add_argument("--deterministic", action="store_true")
     args = ap.parse_args()
     causal = not args.non_causal
     dev = torch.device("cuda:0")
@@ -83,7 +86,10 @@ def main():
 
             def bwd():
                 na.nova_attn_bwd_preprocess(o, do, delta)
-                na.nova_attn_bwd(q, k, v, o, do, lse, delta, dq, dk, dv, cfg.scale, causal, ws)
+                if args.deterministic:
+                    na.nova_attn_bwd_deterministic(q, k, v, do, lse, delta, dq, dk, dv, cfg.scale, causal)
+                else:
+                    na.nova_attn_bwd(q, k, v, o, do, lse, delta, dq, dk, dv, cfg.scale, causal, ws)
 
         t_f, t_b = _time(fwd, args.reps), _time(bwd, args.reps)
         f_flops = cfg.fwd_flops * (1.0 if causal else 2.0)  # the counted figure covers half the square

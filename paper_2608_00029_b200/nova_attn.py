@@ -63,6 +63,8 @@ def load():
     lib.nova_attn_bwd_preprocess_strided.restype = i
     lib.nova_attn_bwd_strided.argtypes = [vp] * 4 + [fp, fp, vp, vp, vp, i, i, i, i] + [sp] * 7 + [f, i, vp, sz, vp]
     lib.nova_attn_bwd_strided.restype = i
+    lib.nova_attn_bwd_deterministic.argtypes = [vp] * 4 + [fp, fp, vp, vp, vp, i, i, i, i, f, i, vp]
+    lib.nova_attn_bwd_deterministic.restype = i
     lib.nova_attn_status_string.argtypes = [i]
     lib.nova_attn_status_string.restype = ctypes.c_char_p
     lib.nova_attn_last_cuda_error.argtypes = []
@@ -257,3 +259,19 @@ def nova_attn_bwd_strided(Q, K, V, dO, LSE, Delta, dQ, dK, dV, scale: float, cau
                                       _stream_ptr(stream))
     if rc != OK:
         raise NovaAttnError(rc, "nova_attn_bwd_strided")
+
+
+def nova_attn_bwd_deterministic(Q, K, V, dO, LSE, Delta, dQ, dK, dV, scale: float, causal: bool = True,
+                                stream=None) -> None:
+    """dQ, dK, dV by the two-kernel backward: bitwise reproducible, no workspace, slower than nova_attn_bwd."""
+    _check_bf16("Q", Q)
+    B, H, T, D = Q.shape
+    for n, t in (("K", K), ("V", V), ("dO", dO), ("dQ", dQ), ("dK", dK), ("dV", dV)):
+        _check_bf16(n, t, Q.shape)
+    _check_f32("LSE", LSE, (B, H, T))
+    _check_f32("Delta", Delta, (B, H, T))
+    rc = load().nova_attn_bwd_deterministic(_ptr(Q), _ptr(K), _ptr(V), _ptr(dO), _ptr(LSE), _ptr(Delta), _ptr(dQ),
+                                            _ptr(dK), _ptr(dV), B, H, T, D, float(scale), int(bool(causal)),
+                                            _stream_ptr(stream))
+    if rc != OK:
+        raise NovaAttnError(rc, "nova_attn_bwd_deterministic")
