@@ -76,6 +76,22 @@ def test_host_side_validation_rejects_before_launch(lib):
     assert e(p, p, p, p, p, p, 1, 1, 16, 64, -2.0, 1, None) == na.ERR_SCALE
 
 
+def test_deterministic_backward_validates_without_a_workspace(lib):
+    from paper_2608_00029_b200 import nova_attn as na
+    p = ctypes.c_void_p(0x1000)
+    odd = ctypes.c_void_p(0x1004)
+    d = lib.nova_attn_bwd_deterministic
+    ptrs = [p] * 9
+    assert d(*ptrs, 0, 1, 16, 64, 1.0, 1, None) == na.ERR_SHAPE
+    assert d(*ptrs, 1, 1, 16, 80, 1.0, 1, None) == na.ERR_UNSUPPORTED
+    assert d(*ptrs, 1, 1, 16, 64, float("nan"), 1, None) == na.ERR_SCALE
+    bad = list(ptrs)
+    bad[6] = None                                        # dQ
+    assert d(*bad, 1, 1, 16, 64, 1.0, 1, None) == na.ERR_NULL
+    bad[6] = odd
+    assert d(*bad, 1, 1, 16, 64, 1.0, 1, None) == na.ERR_ALIGNMENT
+
+
 def test_strided_entry_points_validate_strides(lib):
     from paper_2608_00029_b200 import nova_attn as na
     p = ctypes.c_void_p(0x1000)
