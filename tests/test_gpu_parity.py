@@ -108,6 +108,12 @@ EDGE = [
     (1, 1, 384, 128, False),
     (1, 1, 333, 128, False),
     (3, 1, 640, 64, True),
+    (1, 1, 127, 64, True),      # one short of a tile
+    (1, 1, 128, 128, True),     # exactly one tile: the diagonal tile only
+    (1, 2, 255, 128, False),
+    (40, 8, 64, 64, True),      # many short work items: more items than SMs, one tile each
+    (5, 30, 129, 64, True),     # 150 heads x 2 tiles: item lists of different lengths per CTA, ragged last tile
+    (1, 1, 1537, 64, True),     # 13 tiles, odd length: a single head spread over 13 CTAs in the backward
 ]
 
 

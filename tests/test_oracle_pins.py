@@ -287,3 +287,82 @@ def test_thread_count_does_not_change_results():
             for x, y in zip(a, one):
                 np.testing.assert_array_equal(x[sl], y)
     assert oracle.num_threads() >= 1
+
+
+# ---------------------------------------------------------------------------------------------
+# further invariants: each one fails for a different plausible mistake
+def test_scale_can_be_moved_into_the_queries():
+    """softmax(scale * q.k) only sees the product: scale 0.5 with Q equals scale 1 with Q/2, in O, LSE and dK, dV;
+    dQ picks up the factor of the substitution (dL/dQ = 0.5 * dL/d(Q/2))."""
+    Q, K, V, dO = (rand((1, 2, 7, 4), s) for s in (1, 2, 3, 4))
+    O1, L1 = oracle.attn_fwd(Q, K, V, 0.5, True)
+    O2, L2 = oracle.attn_fwd(0.5 * Q, K, V, 1.0, True)
+    np.testing.assert_allclose(O1, O2, rtol=1e-12, atol=1e-14)
+    np.testing.assert_allclose(L1, L2, rtol=1e-12, atol=1e-14)
+    dQ1, dK1, dV1, D1 = oracle.attn_bwd(Q, K, V, dO, 0.5, True)
+    dQ2, dK2, dV2, D2 = oracle.attn_bwd(0.5 * Q, K, V, dO, 1.0, True)
+    np.testing.assert_allclose(dQ1, 0.5 * dQ2, rtol=1e-11, atol=1e-13)
+    np.testing.assert_allclose(dK1, dK2, rtol=1e-11, atol=1e-13)
+    np.testing.assert_allclose(dV1, dV2, rtol=1e-11, atol=1e-13)
+    np.testing.assert_allclose(D1, D2, rtol=1e-11, atol=1e-13)
+
+
+def test_output_is_linear_in_values_and_dv_is_transposed_probabilities():
+    """O = P V with P independent of V: O(aV1 + bV2) = a O(V1) + b O(V2), LSE does not move, and
+    dV = P^T dO with the P the oracle reports (a transposed or unnormalised P fails here)."""
+    Q, K, V1, V2, dO = (rand((1, 1, 6, 3), s) for s in (11, 12, 13, 14, 15))
+    Oa, La = oracle.attn_fwd(Q, K, V1, 0.7, True)
+    Ob, Lb = oracle.attn_fwd(Q, K, V2, 0.7, True)
+    Oc, Lc = oracle.attn_fwd(Q, K, 2.0 * V1 - 3.0 * V2, 0.7, True)
+    np.testing.assert_allclose(Oc, 2.0 * Oa - 3.0 * Ob, rtol=1e-12, atol=1e-13)
+    np.testing.assert_allclose(Lc, La, rtol=0, atol=0)
+    P = oracle.attn_probs(Q[0, 0], K[0, 0], 0.7, True)   # [T,T] of the one head
+    _, _, dV, _ = oracle.attn_bwd(Q, K, V1, dO, 0.7, True)
+    np.testing.assert_allclose(dV[0, 0], P.T @ dO[0, 0], rtol=1e-12, atol=1e-13)
+    np.testing.assert_allclose(Oa[0, 0], P @ V1[0, 0], rtol=1e-12, atol=1e-13)
+
+
+def test_noncausal_attention_is_equivariant_under_key_permutation():
+    """Without the mask the keys are a set: permuting (K, V) rows together leaves O and LSE alone and
+    permutes dK, dV the same way (an index mix-up between the key loop and the outputs fails here)."""
+    Q, K, V, dO = (rand((1, 2, 9, 5), s) for s in (21, 22, 23, 24))
+    perm = np.random.default_rng(5).permutation(9)
+    O1, L1 = oracle.attn_fwd(Q, K, V, 0.3, False)
+    O2, L2 = oracle.attn_fwd(Q, K[:, :, perm], V[:, :, perm], 0.3, False)
+    np.testing.assert_allclose(O1, O2, rtol=1e-12, atol=1e-13)
+    np.testing.assert_allclose(L1, L2, rtol=1e-12, atol=1e-13)
+    dQ1, dK1, dV1, _ = oracle.attn_bwd(Q, K, V, dO, 0.3, False)
+    dQ2, dK2, dV2, _ = oracle.attn_bwd(Q, K[:, :, perm], V[:, :, perm], dO, 0.3, False)
+    np.testing.assert_allclose(dQ1, dQ2, rtol=1e-11, atol=1e-13)
+    np.testing.assert_allclose(dK1[:, :, perm], dK2, rtol=1e-11, atol=1e-13)
+    np.testing.assert_allclose(dV1[:, :, perm], dV2, rtol=1e-11, atol=1e-13)
+
+
+def test_lse_is_the_potential_of_the_probabilities():
+    """d LSE_i / d k_j = scale * P_ij * q_i (central differences): ties LSE, P and the scale together, and
+    fixes the natural-log base of LSE (a base-2 LSE would be off by ln 2)."""
+    rng = np.random.default_rng(31)
+    Q, K, V = (rng.standard_normal((1, 1, 5, 3)) for _ in range(3))
+    scale, h = 0.8, 1e-6
+    P = oracle.attn_probs(Q[0, 0], K[0, 0], scale, True)
+    for (i, j, d) in ((4, 2, 1), (3, 3, 0), (2, 0, 2), (1, 3, 1)):
+        Kp, Km = K.copy(), K.copy()
+        Kp[0, 0, j, d] += h
+        Km[0, 0, j, d] -= h
+        num = (oracle.attn_fwd(Q, Kp, V, scale, True)[1][0, 0, i] - oracle.attn_fwd(Q, Km, V, scale, True)[1][0, 0, i]) / (2 * h)
+        ana = scale * P[i, j] * Q[0, 0, i, d]  # zero above the diagonal: the masked key cannot move LSE
+        assert abs(num - ana) < 1e-8, (i, j, d, num, ana)
+
+
+def test_heads_and_batches_are_independent():
+    """Every (batch, head) is its own problem: running them together equals running each alone."""
+    Q, K, V, dO = (rand((2, 3, 6, 4), s) for s in (41, 42, 43, 44))
+    O, L = oracle.attn_fwd(Q, K, V, 0.5, True)
+    dQ, dK, dV, D = oracle.attn_bwd(Q, K, V, dO, 0.5, True)
+    for b in range(2):
+        for hd in range(3):
+            sl = (slice(b, b + 1), slice(hd, hd + 1))
+            o, l = oracle.attn_fwd(Q[sl], K[sl], V[sl], 0.5, True)
+            dq, dk, dv, d = oracle.attn_bwd(Q[sl], K[sl], V[sl], dO[sl], 0.5, True)
+            for a, b_ in ((O[sl], o), (L[sl], l), (dQ[sl], dq), (dK[sl], dk), (dV[sl], dv), (D[sl], d)):
+                np.testing.assert_array_equal(a, b_)
