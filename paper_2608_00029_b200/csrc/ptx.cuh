@@ -1,5 +1,5 @@
 // Thin inline-PTX wrappers for the sm_100a features the attention kernels use:
-// mbarrier, TMA (cp.async.bulk.tensor, no cluster multicast anywhere), tcgen05 (TMEM allocation,
+// mbarrier, TMA (cp.async.bulk.tensor; every copy targets this CTA only), tcgen05 (TMEM allocation,
 // UMMA issue/commit, TMEM load/store) and the shared-memory / instruction descriptors of UMMA.
 #pragma once
 
