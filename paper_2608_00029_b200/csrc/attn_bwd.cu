@@ -490,24 +490,39 @@ __device__ __forceinline__ void bwd_compute(uint8_t* smem, BwdBars* bars, uint32
                 if (!ok) break;
                 tc_fence_after();
             }
-            tmem_st_x32(t_p, pk);
-            tmem_wait_st();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&bars->p_ready);
-
             // ---- dS phase: ds = p * (dp - delta); bf16 to TMEM (for dK) and to swizzled smem (for dQ).
             // p is taken from the bf16 pairs already in registers.
             // dP^T of this tile was queued after dQ of the previous one and the tensor pipe completes in
-            // order, so this wait also covers "the previous dQ has finished reading the dS staging buffer".
-            ok = mbar_wait(&bars->dp_full, g & 1, abort_flag);
-            if (!ok) break;
-            tc_fence_after();
+            // order, so the dp_full wait also covers "the previous dQ has finished reading the dS staging
+            // buffer".  Where dP^T never waits for this tile's P^T (kEarlydP) its loads are issued before
+            // the P^T store is awaited, so the two TMEM round trips overlap.
+            constexpr bool kEarlydP = Cfg::kSeparateP && !Cfg::kdQAliased;
             uint32_t dd[32];
             {
                 uint32_t dv[64];
-                tmem_ld_x32(t_dp, dv);
-                tmem_ld_x32(t_dp + 32, dv + 32);
+                if (kEarlydP) {
+                    ok = mbar_wait(&bars->dp_full, g & 1, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    tmem_st_x32(t_p, pk);
+                    tmem_ld_x32(t_dp, dv);
+                    tmem_ld_x32(t_dp + 32, dv + 32);
+                    tmem_wait_st();
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&bars->p_ready);
+                } else {
+                    tmem_st_x32(t_p, pk);
+                    tmem_wait_st();
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&bars->p_ready);
+                    ok = mbar_wait(&bars->dp_full, g & 1, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    tmem_ld_x32(t_dp, dv);
+                    tmem_ld_x32(t_dp + 32, dv + 32);
+                }
                 tmem_wait_ld();
 #pragma unroll
                 for (int x = 0; x < 16; ++x) {
