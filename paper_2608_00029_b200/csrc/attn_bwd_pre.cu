@@ -71,26 +71,43 @@ __global__ void __launch_bounds__(256) bwd_preprocess_kernel(const uint4* __rest
     }
 }
 
+// Each thread takes kConvertItems groups of 8 elements per pass and issues all their loads before the
+// first store.
+constexpr int kConvertItems = 4;
+
 template <bool kContiguous>
 __global__ void __launch_bounds__(256) dq_convert_kernel(const float4* __restrict__ acc, uint4* __restrict__ dQ,
                                                          long long n8, float scale, int lpr_shift, int H, int T,
                                                          const TensorStrides sdq) {
     griddep_launch_dependents();
     griddep_wait();
-    const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
-    for (long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; i < n8; i += stride) {
-        const float4 a = __ldcs(acc + 2 * i);
-        const float4 b = __ldcs(acc + 2 * i + 1);
-        uint4 v;
-        v.x = pack_bf16x2(a.x * scale, a.y * scale);
-        v.y = pack_bf16x2(a.z * scale, a.w * scale);
-        v.z = pack_bf16x2(b.x * scale, b.y * scale);
-        v.w = pack_bf16x2(b.z * scale, b.w * scale);
-        if (kContiguous) {
-            dQ[i] = v;
-        } else {
-            const long long r = i >> lpr_shift;
-            dQ[row_offset16(r, H, T, sdq) + (i - (r << lpr_shift))] = v;
+    const long long stride = static_cast<long long>(gridDim.x) * blockDim.x * kConvertItems;
+    for (long long base = static_cast<long long>(blockIdx.x) * blockDim.x * kConvertItems + threadIdx.x; base < n8;
+         base += stride) {
+        float4 a[kConvertItems], b[kConvertItems];
+#pragma unroll
+        for (int k = 0; k < kConvertItems; ++k) {
+            const long long i = base + static_cast<long long>(k) * blockDim.x;
+            if (i < n8) {
+                a[k] = __ldcs(acc + 2 * i);
+                b[k] = __ldcs(acc + 2 * i + 1);
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < kConvertItems; ++k) {
+            const long long i = base + static_cast<long long>(k) * blockDim.x;
+            if (i >= n8) continue;
+            uint4 v;
+            v.x = pack_bf16x2(a[k].x * scale, a[k].y * scale);
+            v.y = pack_bf16x2(a[k].z * scale, a[k].w * scale);
+            v.z = pack_bf16x2(b[k].x * scale, b[k].y * scale);
+            v.w = pack_bf16x2(b[k].z * scale, b[k].w * scale);
+            if (kContiguous) {
+                dQ[i] = v;
+            } else {
+                const long long r = i >> lpr_shift;
+                dQ[row_offset16(r, H, T, sdq) + (i - (r << lpr_shift))] = v;
+            }
         }
     }
 }
@@ -148,19 +165,17 @@ cudaError_t launch_dq_convert(const float* dq_acc, __nv_bfloat16* dQ, const Attn
                               float scale, int num_sms, cudaStream_t stream) {
     constexpr int kThreads = 256;
     const long long n8 = static_cast<long long>(s.B) * s.H * s.T * s.D / 8;  // D is a multiple of 8
-    long long blocks = (n8 + kThreads - 1) / kThreads;
+    long long blocks = (n8 + kThreads * kConvertItems - 1) / (kThreads * kConvertItems);
     const long long cap = static_cast<long long>(num_sms) * 8;
     if (blocks > cap) blocks = cap;
     if (blocks < 1) blocks = 1;
     const int lpr_shift = (s.D == 64) ? 3 : 4;
     const dim3 grid(static_cast<unsigned>(blocks));
-    if (is_contiguous(s, sdq))
-        return launch_overlapped(dq_convert_kernel<true>, grid, dim3(kThreads), 0, stream,
-                                 reinterpret_cast<const float4*>(dq_acc), reinterpret_cast<uint4*>(dQ), n8, scale,
-                                 lpr_shift, s.H, s.T, sdq);
-    return launch_overlapped(dq_convert_kernel<false>, grid, dim3(kThreads), 0, stream,
-                             reinterpret_cast<const float4*>(dq_acc), reinterpret_cast<uint4*>(dQ), n8, scale, lpr_shift,
-                             s.H, s.T, sdq);
+    auto go = [&](auto kernel) {
+        return launch_overlapped(kernel, grid, dim3(kThreads), 0, stream, reinterpret_cast<const float4*>(dq_acc),
+                                 reinterpret_cast<uint4*>(dQ), n8, scale, lpr_shift, s.H, s.T, sdq);
+    };
+    return is_contiguous(s, sdq) ? go(dq_convert_kernel<true>) : go(dq_convert_kernel<false>);
 }
 
 }  // namespace nova
