@@ -862,6 +862,19 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     tc_fence_after();
     const uint32_t tmem_base = bars->tmem_base;
     griddep_launch_dependents();
+    if (warp == 0 && lane == 0) {  // the first item's K, V and first Q, dO tiles on their way into L2 meanwhile
+        int kt, bh, i0, n_it;
+        if (wl.get(0, &kt, &bh, &i0, &n_it)) {
+            const int head = kStrided ? bh % wl.H : 0, batch = kStrided ? bh / wl.H : 0;
+#pragma unroll
+            for (int h = 0; h < Cfg::kHalves; ++h) {
+                tma_prefetch_tile<kStrided>(&tmK, (wl.orders >> 4) & 15, h * kBoxCols, kt * kBlockK, head, batch, bh);
+                tma_prefetch_tile<kStrided>(&tmQ, wl.orders & 15, h * kBoxCols, i0 * kBlockQ, head, batch, bh);
+                tma_prefetch_tile<kStrided>(&tmV, (wl.orders >> 8) & 15, h * kBoxCols, kt * kBlockK, head, batch, bh);
+                tma_prefetch_tile<kStrided>(&tmdO, (wl.orders >> 12) & 15, h * kBoxCols, i0 * kBlockQ, head, batch, bh);
+            }
+        }
+    }
     griddep_wait();  // everything above overlaps the previous kernel of the stream
 
     if (warp == 0) {

@@ -522,6 +522,19 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     tc_fence_after();
     const uint32_t tmem_base = bars->tmem_base;
     griddep_launch_dependents();
+    if (warp == 0 && lane == 0) {  // the first item's Q tiles and first K, V tiles on their way into L2 meanwhile
+        int blk, bh, n_a, n_b;
+        if (wk.get(0, &blk, &bh, &n_a, &n_b)) {
+            const int head = kStrided ? bh % wk.H : 0, batch = kStrided ? bh / wk.H : 0;
+#pragma unroll
+            for (int h = 0; h < Cfg::kHalves; ++h) {
+                tma_prefetch_tile<kStrided>(&tmK, (wk.orders >> 4) & 15, h * kBoxCols, 0, head, batch, bh);
+                tma_prefetch_tile<kStrided>(&tmQ, wk.orders & 15, h * kBoxCols, blk * kBlockRows, head, batch, bh);
+                tma_prefetch_tile<kStrided>(&tmV, (wk.orders >> 8) & 15, h * kBoxCols, 0, head, batch, bh);
+                tma_prefetch_tile<kStrided>(&tmQ, wk.orders & 15, h * kBoxCols, blk * kBlockRows + kBlockQ, head, batch, bh);
+            }
+        }
+    }
     griddep_wait();  // everything above overlaps the previous kernel of the stream
 
     if (warp == 0) {

@@ -150,6 +150,22 @@ __device__ __forceinline__ void tma_load_tile(void* smem_dst, const CUtensorMap*
         ::"r"(smem_u32(smem_dst)), "l"(m), "r"(smem_u32(bar)), "r"(d), "r"(c1), "r"(c2), "r"(c3)
         : "memory");
 }
+// Asks for the box at the given coordinates to be brought into L2; nothing is written anywhere, so it
+// may run ahead of griddep_wait().
+template <bool kStrided>
+__device__ __forceinline__ void tma_prefetch_tile(const CUtensorMap* m, int order, int d, int t, int h, int b, int bh) {
+    if constexpr (!kStrided) {
+        asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];" ::"l"(m), "r"(d), "r"(t),
+                     "r"(bh)
+                     : "memory");
+        return;
+    }
+    int c1, c2, c3;
+    tma_order_coords(order, t, h, b, c1, c2, c3);
+    asm volatile("cp.async.bulk.prefetch.tensor.4d.L2.global.tile [%0, {%1, %2, %3, %4}];" ::"l"(m), "r"(d), "r"(c1),
+                 "r"(c2), "r"(c3)
+                 : "memory");
+}
 template <bool kStrided>
 __device__ __forceinline__ void tma_store_tile(const CUtensorMap* m, const void* smem_src, int order, int d, int t,
                                                int h, int b, int bh) {
