@@ -427,3 +427,54 @@ def test_random_shapes_and_entry_points(chunk):
         heads = sorted({((i * 7919 + case) % B, (i * 104729 + case) % H) for i in range(min(B * H, 6))})
         ref = h.run_oracle(Q, K, V, dO, scale, causal, heads=heads)
         h.compare(h.select_heads(got, heads), ref, label=label, dO=ref["dO_in"], rms=(T >= 64))
+
+
+def test_two_host_threads_two_streams():
+    """Two host threads drive the library at once, each on its own stream and buffers (different shapes
+    and head dimensions): the calls take the library's lock for the map cache only, the kernels of the
+    two streams share the SMs, and every result is bit-identical to the single-threaded run (dQ within
+    its reduce-order noise)."""
+    import threading
+    from paper_2608_00029_b200 import nova_attn
+    h = _harness()
+    dev = torch.device("cuda:0")
+    cfgs = [W.AttnConfig("mt0", B=2, H=6, T=1024, D=64, seed=811, causal=True),
+            W.AttnConfig("mt1", B=1, H=5, T=700, D=128, seed=812, causal=True)]
+    inputs = [W.make_inputs(c) for c in cfgs]
+    single = [h.run_gpu(*inp, c.scale, True) for inp, c in zip(inputs, cfgs)]
+    results = [None, None]
+    errors = []
+
+    def worker(i):
+        try:
+            cfg = cfgs[i]
+            stream = torch.cuda.Stream(device=dev)
+            with torch.cuda.stream(stream):
+                q, k, v, do = (x.to(dev) for x in inputs[i])
+                shape = (cfg.B, cfg.H, cfg.T, cfg.D)
+                o, dq, dk, dv = (torch.empty(shape, dtype=torch.bfloat16, device=dev) for _ in range(4))
+                lse = torch.empty(shape[:3], dtype=torch.float32, device=dev)
+                delta = torch.empty_like(lse)
+                ws = torch.empty(nova_attn.nova_attn_bwd_workspace_bytes(*shape), dtype=torch.uint8, device=dev)
+                for _ in range(40):
+                    nova_attn.nova_attn_fwd(q, k, v, o, lse, cfg.scale, True, stream=stream)
+                    nova_attn.nova_attn_bwd_preprocess(o, do, delta, stream=stream)
+                    nova_attn.nova_attn_bwd(q, k, v, o, do, lse, delta, dq, dk, dv, cfg.scale, True, ws, stream=stream)
+                stream.synchronize()
+                results[i] = {"O": o.cpu(), "LSE": lse.cpu(), "Delta": delta.cpu(), "dQ": dq.cpu(), "dK": dk.cpu(),
+                              "dV": dv.cpu()}
+        except Exception as e:  # surfaced in the main thread
+            errors.append((i, repr(e)))
+
+    threads = [threading.Thread(target=worker, args=(i,)) for i in range(2)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors, errors
+    nova_attn.nova_attn_poll_device_status()
+    for i in range(2):
+        for name in ("O", "LSE", "Delta", "dK", "dV"):
+            assert torch.equal(results[i][name], single[i][name]), f"thread {i}: {name} differs from the single-threaded run"
+        d = (results[i]["dQ"].float() - single[i]["dQ"].float()).abs().max()
+        assert d <= 1e-2 * single[i]["dQ"].float().abs().max()
