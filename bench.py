@@ -20,6 +20,7 @@ data: weak scaling, no data-path collective.  `--impl reference` times the CPU o
 from __future__ import annotations
 
 import argparse
+import functools
 import json
 import os
 import sys
@@ -240,16 +241,48 @@ def run_ours(args):
     sampler.start()
 
     # ---- device-resident timing
-    for i in range(max(args.warmup, 3)):
-        step(na, cfg, sets[i % n_sets])
+    # One step's five launches (the same C-ABI calls) are recorded once per buffer set into a CUDA graph
+    # and replayed, as a training loop that has captured its step would run them; --launch eager issues
+    # the calls one by one instead.
+    run_step = [functools.partial(step, na, cfg, s) for s in sets]
+    if args.launch == "graph":
+        cap = torch.cuda.Stream(device=dev)
+        with torch.cuda.stream(cap):
+            for f in run_step:
+                f()
+        cap.synchronize()
+        run_step = []
+        for s in sets:
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=cap):
+                step(na, cfg, s)
+            run_step.append(g.replay)
+        # one round over all buffer sets as a single graph: the steps inside keep their programmatic
+        # dependent launch across step boundaries
+        g_round = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g_round, stream=cap):
+            for s in sets:
+                step(na, cfg, s)
+        run_round = g_round.replay
+    else:
+        def run_round():
+            for f in run_step:
+                f()
+
+    def run_steps(n):  # exactly n steps, buffer sets in rotation
+        for _ in range(n // n_sets):
+            run_round()
+        for i in range(n % n_sets):
+            run_step[i]()
+
+    run_steps(max(args.warmup, 3))
     torch.cuda.synchronize()
     multi.barrier()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     torch.cuda.synchronize()
     t_region0 = time.perf_counter()
     ev0.record(stream)
-    for i in range(args.steps):
-        step(na, cfg, sets[i % n_sets])
+    run_steps(args.steps)
     ev1.record(stream)
     torch.cuda.synchronize()
     t_region1 = time.perf_counter()
@@ -378,6 +411,8 @@ def run_ours(args):
                        "T": cfg.T, "D": cfg.D, "causal": True, "parallelism": f"dp{world} (batch split, no collective)",
                        "l2": f"rotating {n_sets} buffer sets of {probe.bytes() / 1e6:.0f} MB "
                              f"({n_sets * probe.bytes() / 1e6:.0f} MB > 126 MB L2)",
+                       "launch": (f"CUDA graph of one round over the {n_sets} buffer sets, replayed (5 kernels per step)"
+                                  if args.launch == "graph" else "eager (5 launches per step)"),
                        "flops_per_step": flops_step, "frac_of_burst_peak": value / world / peaks["bf16_tflops"]},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "ms_per_step": e2e_ms, "steps": e2e_steps},
@@ -399,6 +434,8 @@ def main():
     ap.add_argument("--steps", type=int, default=500)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--launch", choices=["graph", "eager"], default="graph",
+                    help="timed steps replayed from a CUDA graph per buffer set (default) or issued call by call")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)

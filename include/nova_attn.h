@@ -26,6 +26,9 @@
  *     cannot run as built (both indicate a bug or a broken device, never a property of the input), the
  *     kernel records NOVA_ATTN_ERR_TIMEOUT in a device status word, releases what it holds and returns;
  *     nova_attn_poll_device_status() reads the word.
+ *   - Because calls only enqueue, a sequence of them may be captured into a CUDA graph and replayed
+ *     (pointers, shapes and the workspace are baked into the graph); call each entry point once on the
+ *     device before capturing, so that its one-time set-up is not part of the capture.
  *   - Kernels are launched so that each may begin its set-up while the previous kernel in `stream` is
  *     still draining (programmatic dependent launch); each waits for its predecessor before it reads or
  *     writes global memory, so stream order is what the caller observes.

@@ -478,3 +478,44 @@ def test_two_host_threads_two_streams():
             assert torch.equal(results[i][name], single[i][name]), f"thread {i}: {name} differs from the single-threaded run"
         d = (results[i]["dQ"].float() - single[i]["dQ"].float()).abs().max()
         assert d <= 1e-2 * single[i]["dQ"].float().abs().max()
+
+
+def test_cuda_graph_capture_and_replay():
+    """The calls only enqueue work, so a step can be captured into a CUDA graph and replayed (what bench.py
+    times): the replay writes the same O, LSE, Delta, dK, dV bits as the eager calls, and dQ within its
+    reduce-order noise, also when replayed repeatedly."""
+    from paper_2608_00029_b200 import nova_attn
+    dev = torch.device("cuda:0")
+    cfg = W.AttnConfig("graph", B=2, H=5, T=900, D=64, seed=905, causal=True)
+    q, k, v, do = (x.to(dev) for x in W.make_inputs(cfg))
+    shape = (cfg.B, cfg.H, cfg.T, cfg.D)
+    o, dq, dk, dv = (torch.empty(shape, dtype=torch.bfloat16, device=dev) for _ in range(4))
+    lse = torch.empty(shape[:3], dtype=torch.float32, device=dev)
+    delta = torch.empty_like(lse)
+    ws = torch.empty(nova_attn.nova_attn_bwd_workspace_bytes(*shape), dtype=torch.uint8, device=dev)
+
+    def step():
+        nova_attn.nova_attn_fwd(q, k, v, o, lse, cfg.scale, True)
+        nova_attn.nova_attn_bwd_preprocess(o, do, delta)
+        nova_attn.nova_attn_bwd(q, k, v, o, do, lse, delta, dq, dk, dv, cfg.scale, True, ws)
+
+    outs = {"O": o, "LSE": lse, "Delta": delta, "dQ": dq, "dK": dk, "dV": dv}
+    side = torch.cuda.Stream(device=dev)
+    with torch.cuda.stream(side):
+        step()  # also fills the tensor-map cache before the capture
+    side.synchronize()
+    eager = {n: t.clone() for n, t in outs.items()}
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        step()
+        step()
+    for rep in range(3):
+        for n, t in outs.items():
+            t.fill_(float("nan"))
+        graph.replay()
+        torch.cuda.synchronize()
+        nova_attn.nova_attn_poll_device_status()
+        for n in ("O", "LSE", "Delta", "dK", "dV"):
+            assert torch.equal(outs[n], eager[n]), f"replay {rep}: {n} differs from the eager calls"
+        d = (outs["dQ"].float() - eager["dQ"].float()).abs().max()
+        assert d <= 1e-2 * eager["dQ"].float().abs().max()
