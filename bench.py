@@ -245,29 +245,38 @@ def run_ours(args):
     # and replayed, as a training loop that has captured its step would run them; --launch eager issues
     # the calls one by one instead.
     run_step = [functools.partial(step, na, cfg, s) for s in sets]
-    if args.launch == "graph":
+    launch_mode = args.launch
+    eager_step = run_step
+
+    def run_round():
+        for f in eager_step:
+            f()
+
+    if launch_mode == "graph":
         cap = torch.cuda.Stream(device=dev)
         with torch.cuda.stream(cap):
-            for f in run_step:
-                f()
+            run_round()
         cap.synchronize()
-        run_step = []
-        for s in sets:
-            g = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(g, stream=cap):
-                step(na, cfg, s)
-            run_step.append(g.replay)
-        # one round over all buffer sets as a single graph: the steps inside keep their programmatic
-        # dependent launch across step boundaries
-        g_round = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(g_round, stream=cap):
+        try:
+            # thread_local: CUDA calls of other threads (a process group's watchdog) do not end the capture
+            graphs = []
             for s in sets:
-                step(na, cfg, s)
-        run_round = g_round.replay
-    else:
-        def run_round():
-            for f in run_step:
-                f()
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=cap, capture_error_mode="thread_local"):
+                    step(na, cfg, s)
+                graphs.append(g)
+            # one round over all buffer sets as a single graph: the steps inside keep their programmatic
+            # dependent launch across step boundaries
+            g_round = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g_round, stream=cap, capture_error_mode="thread_local"):
+                for s in sets:
+                    step(na, cfg, s)
+            run_step = [g.replay for g in graphs]
+            run_round = g_round.replay
+        except Exception as e:  # the eager calls are the same work: fall back and say so
+            print(f"bench.py: CUDA graph capture failed ({e!r}); timing eager launches", file=sys.stderr)
+            torch.cuda.synchronize()
+            launch_mode = "eager"
 
     def run_steps(n):  # exactly n steps, buffer sets in rotation
         for _ in range(n // n_sets):
@@ -412,7 +421,7 @@ def run_ours(args):
                        "l2": f"rotating {n_sets} buffer sets of {probe.bytes() / 1e6:.0f} MB "
                              f"({n_sets * probe.bytes() / 1e6:.0f} MB > 126 MB L2)",
                        "launch": (f"CUDA graph of one round over the {n_sets} buffer sets, replayed (5 kernels per step)"
-                                  if args.launch == "graph" else "eager (5 launches per step)"),
+                                  if launch_mode == "graph" else "eager (5 launches per step)"),
                        "flops_per_step": flops_step, "frac_of_burst_peak": value / world / peaks["bf16_tflops"]},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "ms_per_step": e2e_ms, "steps": e2e_steps},
