@@ -519,3 +519,71 @@ def test_cuda_graph_capture_and_replay():
             assert torch.equal(outs[n], eager[n]), f"replay {rep}: {n} differs from the eager calls"
         d = (outs["dQ"].float() - eager["dQ"].float()).abs().max()
         assert d <= 1e-2 * eager["dQ"].float().abs().max()
+
+
+def _layout_view(x, kind, rng, dev):
+    """A [B,H,T,D] view with the strides of layout `kind` holding the values of x (storage pre-filled with 7)."""
+    B, H, T, D = x.shape
+    if kind == "bthd":
+        st = torch.empty((B, T, H, D), dtype=x.dtype, device=dev)
+        v = st.permute(0, 2, 1, 3)
+    elif kind == "pad_t":  # padded token stride
+        st = torch.empty((B, H, T, D + 8 * int(rng.integers(1, 5))), dtype=x.dtype, device=dev)
+        v = st[..., :D]
+    elif kind == "pad_h":  # padded head stride
+        st = torch.empty((B, H, T + int(rng.integers(1, 6)), D), dtype=x.dtype, device=dev)
+        v = st[:, :, :T]
+    elif kind == "hbtd":   # heads outermost
+        st = torch.empty((H, B, T, D), dtype=x.dtype, device=dev)
+        v = st.permute(1, 0, 2, 3)
+    elif kind == "tbhd":   # tokens outermost
+        st = torch.empty((T, B, H, D), dtype=x.dtype, device=dev)
+        v = st.permute(1, 2, 0, 3)
+    else:
+        st = torch.empty((B, H, T, D), dtype=x.dtype, device=dev)
+        v = st
+    st.fill_(7.0)
+    v.copy_(x)
+    return v, st
+
+
+def test_random_tensor_layouts():
+    """Every bf16 tensor of the strided entry points in a layout of its own (plain, [B,T,H,D], padded token
+    or head stride, heads or tokens outermost), 60 seeded cases: only addressing changes, so O, LSE, Delta,
+    dK, dV are bit-identical to the plain entry points, dQ within its reduce-order noise, and nothing is
+    written between the rows of a padded output."""
+    from paper_2608_00029_b200 import nova_attn
+    dev = torch.device("cuda:0")
+    rng = np.random.default_rng(4242)
+    kinds = ["bhtd", "bthd", "pad_t", "pad_h", "hbtd", "tbhd"]
+    for case in range(60):
+        D = int(rng.choice([64, 128]))
+        T = int(rng.choice([1, 5, 64, 127, 128, 129, 200, 256, 300, 511, 640, 1000]))
+        B, H = int(rng.integers(1, 4)), int(rng.integers(1, 6))
+        causal = bool(rng.random() < 0.7)
+        scale = D ** -0.5
+        g = torch.Generator().manual_seed(4242 + case)
+        q, k, v, do = (torch.randn(B, H, T, D, generator=g).to(torch.bfloat16).to(dev) for _ in range(4))
+        o, dq, dk, dv = (torch.empty((B, H, T, D), dtype=torch.bfloat16, device=dev) for _ in range(4))
+        lse = torch.empty((B, H, T), dtype=torch.float32, device=dev)
+        delta = torch.empty_like(lse)
+        nova_attn.nova_attn_fwd(q, k, v, o, lse, scale, causal)
+        nova_attn.nova_attn_bwd_preprocess(o, do, delta)
+        nova_attn.nova_attn_bwd(q, k, v, o, do, lse, delta, dq, dk, dv, scale, causal)
+        ks = [str(rng.choice(kinds)) for _ in range(8)]
+        (q_v, _), (k_v, _), (v_v, _), (do_v, _) = (_layout_view(x, kd, rng, dev) for x, kd in zip((q, k, v, do), ks[:4]))
+        outs = [_layout_view(torch.full_like(q, 7.0), kd, rng, dev) for kd in ks[4:]]
+        (o_v, o_st), (dq_v, dq_st), (dk_v, dk_st), (dv_v, dv_st) = outs
+        lse2, delta2 = torch.empty_like(lse), torch.empty_like(delta)
+        nova_attn.nova_attn_fwd_strided(q_v, k_v, v_v, o_v, lse2, scale, causal)
+        nova_attn.nova_attn_bwd_preprocess_strided(o_v, do_v, delta2)
+        nova_attn.nova_attn_bwd_strided(q_v, k_v, v_v, do_v, lse2, delta2, dq_v, dk_v, dv_v, scale, causal)
+        nova_attn.nova_attn_poll_device_status()
+        label = f"layouts case {case} B={B} H={H} T={T} D={D} causal={causal} {ks}: "
+        for name, a, b in (("O", o_v, o), ("LSE", lse2, lse), ("Delta", delta2, delta), ("dK", dk_v, dk), ("dV", dv_v, dv)):
+            assert torch.equal(a.contiguous(), b), label + name + " differs from the plain entry points"
+        d = (dq_v.float() - dq.float()).abs().max()
+        assert d <= 1e-2 * max(float(dq.float().abs().max()), 1e-3), label + "dQ"
+        for name, view, st in (("O", o_v, o_st), ("dQ", dq_v, dq_st), ("dK", dk_v, dk_st), ("dV", dv_v, dv_st)):
+            view.fill_(7.0)  # what is left must be the untouched padding
+            assert bool((st == 7.0).all()), label + name + ": write outside the rows of the view"
