@@ -485,11 +485,6 @@ __device__ __forceinline__ void bwd_compute(uint8_t* smem, BwdBars* bars, uint32
                 else
                     bwd_p_phase<false>(sv, s_lse4, c, pk, true, false, r, 64 * half);
             }
-            if (Cfg::kSeparateP && g > 0) {  // dV of the previous tile must be done reading the P^T columns
-                ok = mbar_wait(&bars->do_empty[(g - 1) % Cfg::kdOStages], ((g - 1) / Cfg::kdOStages) & 1, abort_flag);
-                if (!ok) break;
-                tc_fence_after();
-            }
             // ---- dS phase: ds = p * (dp - delta); bf16 to TMEM (for dK) and to swizzled smem (for dQ).
             // p is taken from the bf16 pairs already in registers.
             // dP^T of this tile was queued after dQ of the previous one and the tensor pipe completes in
@@ -497,10 +492,13 @@ __device__ __forceinline__ void bwd_compute(uint8_t* smem, BwdBars* bars, uint32
             // buffer".  Where dP^T never waits for this tile's P^T (kEarlydP) its loads are issued before
             // the P^T store is awaited, so the two TMEM round trips overlap.
             constexpr bool kEarlydP = Cfg::kSeparateP && !Cfg::kdQAliased;
+            static_assert(kEarlydP || !Cfg::kSeparateP, "P^T columns of their own need the dp_full wait below");
             uint32_t dd[32];
             {
                 uint32_t dv[64];
                 if (kEarlydP) {
+                    // dP^T of this tile was queued after dV of the previous one and the tensor pipe completes
+                    // in order, so this wait also covers "dV has finished reading the P^T columns".
                     ok = mbar_wait(&bars->dp_full, g & 1, abort_flag);
                     if (!ok) break;
                     tc_fence_after();
