@@ -57,8 +57,11 @@ struct BwdCfg {
     static constexpr int kdOStages = (D == 64) ? 2 : 1;
     static constexpr int kOffK = 0;                                   // kKVStages x K tile
     static constexpr int kOffV = kKVStages * kTileBytes;              // kKVStages x V tile
-    static constexpr int kOffQ = 2 * kKVStages * kTileBytes;          // 2 stages
-    static constexpr int kOffdO = kOffQ + 2 * kTileBytes;             // kdOStages stages
+    // Three Q stages where shared memory has room: a Q tile is requested two tiles ahead, so that S^T of
+    // the next tile never waits for it.
+    static constexpr int kQStages = (D == 64) ? 3 : 2;
+    static constexpr int kOffQ = 2 * kKVStages * kTileBytes;          // kQStages stages
+    static constexpr int kOffdO = kOffQ + kQStages * kTileBytes;      // kdOStages stages
     static constexpr int kOffdS = kOffdO + kdOStages * kTileBytes;    // [2 query halves][128 keys][64 queries] bf16
     static constexpr int kOffRow = kOffdS + 2 * kHalfTileBytes;       // 2 x (-LSE*log2e[128], -Delta[128]) fp32
     // Staging buffer of the dQ warps: two boxes of [128 rows x 128 bytes], 128-byte swizzled like every
@@ -87,7 +90,7 @@ struct BwdCfg {
 
 struct BwdBars {
     uint64_t kv_full[2], kv_empty[2];
-    uint64_t q_full[2], q_empty[2];
+    uint64_t q_full[3], q_empty[3];
     uint64_t do_full[2], do_empty[2];
     uint64_t s_full, dp_full;         // UMMA -> compute
     uint64_t p_ready, ds_ready;       // compute (one arrival per warp) -> UMMA
@@ -126,7 +129,7 @@ __device__ __forceinline__ void bwd_producer(const CUtensorMap* tmQ, const CUten
                                              const WorkList& wl) {
     using Cfg = BwdCfg<D>;
     volatile int* abort_flag = &bars->abort_flag;
-    int armed_kv[2] = {-1, -1}, armed_q[2] = {-1, -1}, armed_do[2] = {-1, -1};
+    int armed_kv[2] = {-1, -1}, armed_q[3] = {-1, -1, -1}, armed_do[2] = {-1, -1};
     bool ok = true;
     int w = 0, g = 0;  // items and query tiles processed so far by this CTA
     for (int p = 0; p < wl.passes() && ok; ++p) {
@@ -147,12 +150,12 @@ __device__ __forceinline__ void bwd_producer(const CUtensorMap* tmQ, const CUten
                           (wl.orders >> 8) & 15, h * kBoxCols, kt * kBlockK, head, batch, bh);
         }
         for (int it = 0; it < n_it; ++it, ++g) {
-            const int st = g & 1;
+            const int st = g % Cfg::kQStages;
             const int qrow = (i0 + it) * kBlockQ;
-            ok = mbar_wait(&bars->q_empty[st], ((g >> 1) & 1) ^ 1, abort_flag);
+            ok = mbar_wait(&bars->q_empty[st], ((g / Cfg::kQStages) & 1) ^ 1, abort_flag);
             if (!ok) break;
             mbar_expect_tx(&bars->q_full[st], Cfg::kTileBytes);
-            armed_q[st] = (g >> 1) & 1;
+            armed_q[st] = (g / Cfg::kQStages) & 1;
 #pragma unroll
             for (int h = 0; h < Cfg::kHalves; ++h)
                 tma_load_tile<kStrided>(smem + Cfg::kOffQ + st * Cfg::kTileBytes + h * kHalfTileBytes, tmQ, &bars->q_full[st],
@@ -175,9 +178,10 @@ __device__ __forceinline__ void bwd_producer(const CUtensorMap* tmQ, const CUten
         int none = 0;
         for (int s = 0; s < 2; ++s) {
             if (armed_kv[s] >= 0) (void)mbar_wait(&bars->kv_full[s], armed_kv[s], &none);
-            if (armed_q[s] >= 0) (void)mbar_wait(&bars->q_full[s], armed_q[s], &none);
             if (armed_do[s] >= 0) (void)mbar_wait(&bars->do_full[s], armed_do[s], &none);
         }
+        for (int s = 0; s < Cfg::kQStages; ++s)
+            if (armed_q[s] >= 0) (void)mbar_wait(&bars->q_full[s], armed_q[s], &none);
     }
 }
 
@@ -195,11 +199,13 @@ __device__ __forceinline__ void bwd_mma(uint8_t* smem, BwdBars* bars, uint32_t t
     // is added.  "_k": read K-major (rows of the operand are its M/N index), "_m": read MN-major (rows
     // are its K index; LBO = distance between 64-element halves).
     const uint32_t hi = umma_desc_hi_sw128(1024);
-    uint32_t q_k[2], q_m[2], do_k[2], do_m[2];
+    // Q stage st: the address field counts 16-byte units, so a stage is kTileBytes / 16 further on.
+    const uint32_t q_k0 = umma_desc_lo(smem_u32(smem + Cfg::kOffQ), 16);
+    const uint32_t q_m0 = umma_desc_lo(smem_u32(smem + Cfg::kOffQ), kHalfTileBytes);
+    constexpr uint32_t kQStageStep = Cfg::kTileBytes >> 4;
+    uint32_t do_k[2], do_m[2];
 #pragma unroll
     for (int st = 0; st < 2; ++st) {
-        q_k[st] = umma_desc_lo(smem_u32(smem + Cfg::kOffQ + st * Cfg::kTileBytes), 16);
-        q_m[st] = umma_desc_lo(smem_u32(smem + Cfg::kOffQ + st * Cfg::kTileBytes), kHalfTileBytes);
         do_k[st] = umma_desc_lo(smem_u32(smem + Cfg::kOffdO + (st % Cfg::kdOStages) * Cfg::kTileBytes), 16);
         do_m[st] = umma_desc_lo(smem_u32(smem + Cfg::kOffdO + (st % Cfg::kdOStages) * Cfg::kTileBytes), kHalfTileBytes);
     }
@@ -208,8 +214,8 @@ __device__ __forceinline__ void bwd_mma(uint8_t* smem, BwdBars* bars, uint32_t t
     // The whole warp runs this role in uniform control flow; one elected lane issues.
     const bool el = elect_one();
 
-    auto issue_st = [&](int gq, uint32_t kd) {  // S^T = K Q^T: K tile `kd`, query tile in Q stage gq & 1
-        const uint32_t b = q_k[gq & 1];
+    auto issue_st = [&](int gq, uint32_t kd) {  // S^T = K Q^T: K tile `kd`, query tile in Q stage gq % kQStages
+        const uint32_t b = q_k0 + (gq % Cfg::kQStages) * kQStageStep;
         if (el) {
 #pragma unroll
             for (int k = 0; k < D / 16; ++k) {
@@ -252,7 +258,7 @@ __device__ __forceinline__ void bwd_mma(uint8_t* smem, BwdBars* bars, uint32_t t
         k_m = umma_desc_lo(smem_u32(smem + Cfg::kOffK + ks * Cfg::kTileBytes), kHalfTileBytes);
         v_k = umma_desc_lo(smem_u32(smem + Cfg::kOffV + ks * Cfg::kTileBytes), 16);
         ok = mbar_wait(&bars->kv_full[ks], (w / Cfg::kKVStages) & 1, abort_flag);
-        if (ok) ok = mbar_wait(&bars->q_full[g & 1], (g >> 1) & 1, abort_flag);
+        if (ok) ok = mbar_wait(&bars->q_full[g % Cfg::kQStages], (g / Cfg::kQStages) & 1, abort_flag);
         if (ok && Cfg::kdQAliased && g > 0 && !wl.no_dq) ok = mbar_wait(&bars->dq_free, (g - 1) & 1, abort_flag);
         if (ok) ok = mbar_wait(&bars->do_full[g % Cfg::kdOStages], (g / Cfg::kdOStages) & 1, abort_flag);
         if (!ok) break;
@@ -265,7 +271,6 @@ __device__ __forceinline__ void bwd_mma(uint8_t* smem, BwdBars* bars, uint32_t t
         }
         first_queued = false;
         for (int it = 0; it < n_it && ok; ++it, ++g) {
-            const int st = g & 1;
             const bool more = it + 1 < n_it;
             const bool cross = !more && has_next && Cfg::kSeparateP && !Cfg::kdQAliased;  // next tile opens the next item
             ok = mbar_wait(&bars->p_ready, g & 1, abort_flag);
@@ -273,7 +278,7 @@ __device__ __forceinline__ void bwd_mma(uint8_t* smem, BwdBars* bars, uint32_t t
             tc_fence_after();
             if (Cfg::kSeparateP && (more || cross)) {  // S^T columns are free as soon as the compute warps have read them
                 if (cross) ok = mbar_wait(&bars->kv_full[ks_n], ((w + 1) / Cfg::kKVStages) & 1, abort_flag);
-                if (ok) ok = mbar_wait(&bars->q_full[st ^ 1], ((g + 1) >> 1) & 1, abort_flag);
+                if (ok) ok = mbar_wait(&bars->q_full[(g + 1) % Cfg::kQStages], ((g + 1) / Cfg::kQStages) & 1, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
                 issue_st(g + 1, cross ? k_k_n : k_k);
@@ -294,7 +299,7 @@ __device__ __forceinline__ void bwd_mma(uint8_t* smem, BwdBars* bars, uint32_t t
             }
             __syncwarp();
             if (!Cfg::kSeparateP && more) {  // P^T lives in the S^T columns: dV must be queued first
-                ok = mbar_wait(&bars->q_full[st ^ 1], ((g + 1) >> 1) & 1, abort_flag);
+                ok = mbar_wait(&bars->q_full[(g + 1) % Cfg::kQStages], ((g + 1) / Cfg::kQStages) & 1, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
                 issue_st(g + 1, k_k);
@@ -303,12 +308,12 @@ __device__ __forceinline__ void bwd_mma(uint8_t* smem, BwdBars* bars, uint32_t t
             if (!ok) break;
             tc_fence_after();
             if (el) {
-                const uint32_t b = q_m[st];
+                const uint32_t b = q_m0 + (g % Cfg::kQStages) * kQStageStep;
 #pragma unroll
                 for (int k = 0; k < kBlockQ / 16; ++k)
                     umma_ts(t_dk, t_dp + (k / 4) * 64 + (k % 4) * 8, umma_desc_join(b + k * 128, hi), kIdescKV,
                             (it > 0 || k > 0) ? 1u : 0u);
-                tc_commit(&bars->q_empty[st]);
+                tc_commit(&bars->q_empty[g % Cfg::kQStages]);
             }
             __syncwarp();
             // dQ_i = dS K_j, 64 head-dim columns per accumulator half; 16 keys per instruction.
@@ -825,6 +830,10 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             mbar_init(&bars->kv_empty[s], 1);
             mbar_init(&bars->q_full[s], 1);
             mbar_init(&bars->q_empty[s], 1);
+            if (s == 0) {
+                mbar_init(&bars->q_full[2], 1);
+                mbar_init(&bars->q_empty[2], 1);
+            }
             mbar_init(&bars->do_full[s], 1);
             mbar_init(&bars->do_empty[s], 1);
             mbar_init(&bars->row_full[s], 2);
