@@ -2,6 +2,8 @@
 """Benchmark of the fused causal attention path (forward + backward preprocess + backward).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+    python bench.py --workload long_context --profile --steps 1 --warmup 1     (a short run to put under ncu)
+    python bench.py --grid causal|noncausal|fused|deterministic                (the paper's shape ranges)
 
 One step = nova_attn_fwd + nova_attn_bwd_preprocess + nova_attn_bwd over one batch of the GPT-2-small
 training attention shape (B=8, H=12, T=1024, D=64, causal, bf16).  Prints ONE JSON line.
@@ -10,8 +12,10 @@ training attention shape (B=8, H=12, T=1024, D=64, causal, bf16).  Prints ONE JS
              HBM, timed with CUDA events on the launching stream, max over ranks.
   e2e        the same metric with the step's inputs copied from pinned host memory and its results
              copied back inside the timed region.
-  roofline   tensor-core roofline of the dominant kernel (the fused backward), from a second pass
-             that brackets each kernel with events.
+  roofline   tensor-core roofline of the dominant kernel (the fused backward) against the measured burst
+             bf16 peak, from a second pass that brackets each kernel with events, and the forward and the
+             whole backward (preprocess + clear + main + convert, timed in sequence) against the targets of
+             50 % and 35 % of that peak.
   cpu_baseline  the fp64 oracle timed on the host cores on a bounded sample of the same workload.
 
 With N > 1 (launched by torchrun, one rank per GPU) every rank runs the same per-GPU batch on its own
@@ -155,7 +159,7 @@ def run_reference(args):
         return 0
     import oracle
     oracle.build()
-    cfg = W.CONFIGS[WORKLOAD]
+    cfg = W.CONFIGS[args.workload]
     Q, K, V, dO = W.make_inputs(cfg)
     threads = oracle.num_threads()
 
@@ -214,6 +218,126 @@ def step(na, cfg, s):
     na.nova_attn_bwd(s.q, s.k, s.v, s.o, s.do, s.lse, s.delta, s.dq, s.dk, s.dv, cfg.scale, cfg.causal, s.ws)
 
 
+def run_profile(args, na, cfg, dev):
+    """A short run of the step on one buffer set, nothing else: the command to put under a profiler."""
+    s = BufferSet(cfg, dev, W.make_inputs(cfg))
+    for _ in range(args.warmup + args.steps):
+        step(na, cfg, s)
+    na.nova_attn_poll_device_status()
+    print(json.dumps({"profile_run": cfg.name, "B": cfg.B, "H": cfg.H, "T": cfg.T, "D": cfg.D,
+                      "steps": args.warmup + args.steps, "checksum": float(s.dq.float().sum())}), flush=True)
+    return 0
+
+
+# The eight shapes of the grid lie inside the ranges of the paper's attention microbenchmark (Section 6.1:
+# sequence lengths 512 to 2048, 12 to 32 heads, head dimension 64 or 128; the per-shape values are in a
+# figure), at batch 16 like that figure's "16x12x64" label.
+GRID = [(512, 12, 64), (1024, 12, 64), (2048, 12, 64), (1024, 16, 64), (1024, 20, 64), (512, 32, 128),
+        (1024, 32, 128), (2048, 32, 128)]  # (T, H, D)
+
+
+class GridSet:
+    """One set of buffers for a grid shape, plain [B,H,T,D] or the fused-projection layout (Q, K, V read in
+    place from [B,T,3,H,D], O / dO as [B,T,H,D], dQ, dK, dV written into one [B,T,3,H,D] buffer)."""
+
+    def __init__(self, na, cfg, dev, inputs, fused):
+        B, H, T, D = cfg.B, cfg.H, cfg.T, cfg.D
+        q, k, v, do = (x.to(dev) for x in inputs)
+        self.lse = torch.empty((B, H, T), dtype=torch.float32, device=dev)
+        self.delta = torch.empty_like(self.lse)
+        self.ws = torch.empty(na.nova_attn_bwd_workspace_bytes(B, H, T, D), dtype=torch.uint8, device=dev)
+        if fused:
+            qkv = torch.empty((B, T, 3, H, D), dtype=torch.bfloat16, device=dev)
+            for i, x in enumerate((q, k, v)):
+                qkv[:, :, i] = x.permute(0, 2, 1, 3)
+            dqkv = torch.empty_like(qkv)
+            self.keep = (qkv, dqkv)
+            self.q, self.k, self.v = (qkv[:, :, i].permute(0, 2, 1, 3) for i in range(3))
+            self.dq, self.dk, self.dv = (dqkv[:, :, i].permute(0, 2, 1, 3) for i in range(3))
+            self.o = torch.empty((B, T, H, D), dtype=torch.bfloat16, device=dev).permute(0, 2, 1, 3)
+            self.do = do.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+        else:
+            self.q, self.k, self.v, self.do = q, k, v, do
+            self.o, self.dq, self.dk, self.dv = (torch.empty_like(q) for _ in range(4))
+        self.nbytes = 8 * q.numel() * 2 + 2 * self.lse.numel() * 4 + self.ws.numel()
+
+
+def run_grid(args):
+    """Forward and backward (preprocess + backward) timed over the grid through the same protocol as the
+    headline number: buffer sets in rotation so that no call finds its inputs in L2, warm-up, CUDA events
+    on the launching stream around `--steps` calls issued one by one, clocks sampled meanwhile.  Prints a
+    markdown table and one JSON line with the rows and the clock record."""
+    from paper_2608_00029_b200 import nova_attn as na
+    na.load()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the attention path has no CPU fallback")
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    stream = torch.cuda.current_stream()
+    mode = args.grid
+    causal = mode != "noncausal"
+    fused, det = mode == "fused", mode == "deterministic"
+    sampler = ClockSampler(0)
+    sampler.start()
+    t_region0 = time.perf_counter()
+    rows = []
+    print("| B | H | T | D | causal | fwd ms | fwd TFLOP/s | bwd ms | bwd TFLOP/s | fwd+bwd ms |", file=sys.stderr)
+    print("|---|---|---|---|---|---|---|---|---|---|", file=sys.stderr)
+    for T, H, D in GRID:
+        cfg = W.AttnConfig(f"grid_T{T}_H{H}_D{D}", B=args.grid_batch, H=H, T=T, D=D, seed=5, causal=causal)
+        first = GridSet(na, cfg, dev, W.make_inputs(cfg), fused)
+        n_sets = max(2, int(L2_BYTES * 2 // first.nbytes) + 2)
+        sets = [first] + [GridSet(na, cfg, dev, W.make_inputs(cfg, seed=5 + i), fused) for i in range(1, n_sets)]
+
+        def fwd(s):
+            if fused:
+                na.nova_attn_fwd_strided(s.q, s.k, s.v, s.o, s.lse, cfg.scale, causal)
+            else:
+                na.nova_attn_fwd(s.q, s.k, s.v, s.o, s.lse, cfg.scale, causal)
+
+        def bwd(s):
+            if fused:
+                na.nova_attn_bwd_preprocess_strided(s.o, s.do, s.delta)
+                na.nova_attn_bwd_strided(s.q, s.k, s.v, s.do, s.lse, s.delta, s.dq, s.dk, s.dv, cfg.scale, causal, s.ws)
+                return
+            na.nova_attn_bwd_preprocess(s.o, s.do, s.delta)
+            if det:
+                na.nova_attn_bwd_deterministic(s.q, s.k, s.v, s.do, s.lse, s.delta, s.dq, s.dk, s.dv, cfg.scale, causal)
+            else:
+                na.nova_attn_bwd(s.q, s.k, s.v, s.o, s.do, s.lse, s.delta, s.dq, s.dk, s.dv, cfg.scale, causal, s.ws)
+
+        def timed(fn):
+            for i in range(max(args.warmup, 3)):
+                fn(sets[i % n_sets])
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for i in range(args.steps):
+                fn(sets[i % n_sets])
+            e1.record(stream)
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1) / args.steps
+
+        for s in sets:  # every set holds a valid O, LSE, Delta before the backward is timed
+            fwd(s)
+        t_f, t_b = timed(fwd), timed(bwd)
+        na.nova_attn_poll_device_status()
+        f_flops = cfg.fwd_flops * (1.0 if causal else 2.0)  # the counted figure covers half the square
+        row = {"B": cfg.B, "H": H, "T": T, "D": D, "causal": causal, "fwd_ms": t_f, "fwd_tflops": f_flops / t_f / 1e9,
+               "bwd_ms": t_b, "bwd_tflops": 2.5 * f_flops / t_b / 1e9, "buffer_sets": n_sets}
+        rows.append(row)
+        print(f"| {cfg.B} | {H} | {T} | {D} | {'yes' if causal else 'no'} | {t_f:.4f} | {row['fwd_tflops']:.0f} | "
+              f"{t_b:.4f} | {row['bwd_tflops']:.0f} | {t_f + t_b:.4f} |", file=sys.stderr, flush=True)
+        del sets, first
+        torch.cuda.empty_cache()
+    sampler.stop()
+    sampler.join(timeout=2)
+    print(json.dumps({"grid": mode, "steps": args.steps, "warmup": max(args.warmup, 3), "launch": "eager",
+                      "l2": "buffer sets in rotation, more than twice the 126 MB L2 between two uses of a set",
+                      "rows": rows, "clocks": sampler.summary(t_region0, time.perf_counter())}), flush=True)
+    return 0
+
+
 def run_ours(args):
     from paper_2608_00029_b200 import nova_attn as na
     na.load()  # fails loudly if the CUDA library has not been built
@@ -226,9 +350,11 @@ def run_ours(args):
         multi.init_process_group("nccl")
     peaks, peak_src = load_peaks()
 
-    base = W.CONFIGS[WORKLOAD]
+    base = W.CONFIGS[args.workload]
     plan = multi.weak_scaling_plan(base.B, world, rank)
     cfg = base.replace(B=plan["local_batch"])
+    if args.profile:
+        return run_profile(args, na, cfg, dev)
     # Rotate over enough independent buffer sets that the data touched between two uses of the same
     # set exceeds L2, so no step finds its inputs cached from the previous use.
     probe = BufferSet(cfg, dev, W.make_inputs(cfg, seed=base.seed + 1000 * rank))
@@ -319,29 +445,60 @@ def run_ours(args):
             e[3 + n].record(stream)
     torch.cuda.synchronize()
     kernel_ms = {n: sum(e[i].elapsed_time(e[i + 1]) for e in evs) / k_steps for i, n in enumerate(names)}
+
+    # ---- forward, and the whole backward as one sequence (preprocess + clear + main + convert), each
+    # bracketed by events: what the 50 % / 35 % targets are stated on
+    evq = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(k_steps)]
+    for i in range(k_steps):
+        s = sets[i % n_sets]
+        e = evq[i]
+        e[0].record(stream)
+        na.nova_attn_fwd(s.q, s.k, s.v, s.o, s.lse, cfg.scale, cfg.causal)
+        e[1].record(stream)
+        na.nova_attn_bwd_preprocess(s.o, s.do, s.delta)
+        na.nova_attn_bwd(s.q, s.k, s.v, s.o, s.do, s.lse, s.delta, s.dq, s.dk, s.dv, cfg.scale, cfg.causal, s.ws)
+        e[2].record(stream)
+    torch.cuda.synchronize()
+    fwd_seq_ms = sum(e[0].elapsed_time(e[1]) for e in evq) / k_steps
+    bwd_seq_ms = sum(e[1].elapsed_time(e[2]) for e in evq) / k_steps
+
     bwd_ms = kernel_ms["bwd_main"]
     achieved = cfg.bwd_flops / (bwd_ms * 1e-3) / 1e12
-    # a kernel timed inside a long back-to-back run is compared with the sustained GEMM figure
-    peak = peaks["bf16_tflops_sustained"]
+    # every launch of these passes is timed on its own, between events, at full clocks: the burst figure
+    # is the peak that applies; the sustained one is given beside it
+    peak = peaks["bf16_tflops"]
+    fwd_tflops = cfg.fwd_flops / (fwd_seq_ms * 1e-3) / 1e12
+    bwd_tflops = cfg.bwd_flops / (bwd_seq_ms * 1e-3) / 1e12
     roofline = {
         "bound": "tensor", "kernel": "attn_bwd_kernel", "achieved": achieved, "peak": peak, "unit": UNIT,
-        "frac": achieved / peak, "traffic": None, "peak_source": f"{peak_src} bf16_tflops_sustained",
-        "frac_of_burst_peak": achieved / peaks["bf16_tflops"], "ms_per_launch": bwd_ms,
+        "frac": achieved / peak, "traffic": None, "traffic_source": None,
+        "peak_source": f"{peak_src} bf16_tflops (burst)",
+        "peak_sustained": peaks["bf16_tflops_sustained"],
+        "frac_of_sustained_peak": achieved / peaks["bf16_tflops_sustained"], "ms_per_launch": bwd_ms,
         "kernel_ms": kernel_ms,
-        "fwd_tflops": cfg.fwd_flops / (kernel_ms["fwd"] * 1e-3) / 1e12,
-        "fwd_frac_of_burst_peak": cfg.fwd_flops / (kernel_ms["fwd"] * 1e-3) / 1e12 / peaks["bf16_tflops"],
+        "targets": {
+            "fwd": {"what": "nova_attn_fwd", "ms": fwd_seq_ms, "tflops": fwd_tflops, "frac": fwd_tflops / peak,
+                    "target": 0.50},
+            "bwd": {"what": "nova_attn_bwd_preprocess + nova_attn_bwd (clear, main, convert) in sequence",
+                    "ms": bwd_seq_ms, "tflops": bwd_tflops, "frac": bwd_tflops / peak, "target": 0.35},
+        },
         "preprocess_gbs": (4.0 * cfg.B * cfg.H * cfg.T * cfg.D + 4.0 * cfg.B * cfg.H * cfg.T)
         / (kernel_ms["bwd_preprocess"] * 1e-3) / 1e9,
+        "preprocess_frac_of_hbm_peak": (4.0 * cfg.B * cfg.H * cfg.T * cfg.D + 4.0 * cfg.B * cfg.H * cfg.T)
+        / (kernel_ms["bwd_preprocess"] * 1e-3) / 1e9 / peaks["hbm_gbs"],
     }
-    # DRAM bytes of one launch of the dominant kernel, from the committed ncu summary of this workload
-    # (a "traffic_bytes_per_launch: N" line); absent or another workload -> null.
-    traffic_path = os.path.join(ROOT, "profiles", f"attn_bwd_kernel_{base.name}.md")
+    # DRAM bytes of one launch of the dominant kernel are not measured by this run: they come from the
+    # committed ncu summary of this workload (its "traffic_bytes_per_launch: N" line); absent or another
+    # workload -> null.
+    traffic_rel = os.path.join("profiles", f"attn_bwd_kernel_{base.name}.md")
+    traffic_path = os.path.join(ROOT, traffic_rel)
     if os.path.exists(traffic_path) and cfg.B == base.B:
         try:
             with open(traffic_path) as f:
                 for line in f:
                     if line.startswith("traffic_bytes_per_launch:"):
                         roofline["traffic"] = int(line.split(":")[1])
+                        roofline["traffic_source"] = f"{traffic_rel} (committed ncu summary, not measured in this run)"
         except Exception:
             pass
 
@@ -445,7 +602,18 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--launch", choices=["graph", "eager"], default="graph",
                     help="timed steps replayed from a CUDA graph per buffer set (default) or issued call by call")
+    ap.add_argument("--workload", choices=W.CONFIG_ORDER, default=WORKLOAD,
+                    help="the configuration to run (the headline number is quoted on the default)")
+    ap.add_argument("--profile", action="store_true",
+                    help="only run warmup + steps steps on one buffer set and exit: a short command for a profiler")
+    ap.add_argument("--grid", choices=["causal", "noncausal", "fused", "deterministic"], default=None,
+                    help="time forward and backward over the paper's shape ranges instead of the headline workload")
+    ap.add_argument("--grid-batch", type=int, default=16)
     args = ap.parse_args()
+    if args.grid:
+        if args.steps == 500:
+            args.steps = 30
+        return run_grid(args)
     if args.impl == "reference":
         return run_reference(args)
     return run_ours(args)

@@ -148,15 +148,21 @@ int nova_attn_bwd_steps(const void* Q, const void* K, const void* V, const void*
  *   - The array holds nova_attn_static_scratch_bytes() = 32 MiB, i.e. B*H*T*D <= 8 Mi elements (the
  *     GPT-2-small training shape B=8, H=12, T=1024, D=64 fits).  Larger problems are rejected with
  *     NOVA_ATTN_ERR_WORKSPACE before anything is launched; use nova_attn_bwd for those.
- *   - The array is part of the library image: every GPU that loads the library holds the 32 MiB until
- *     the process exits, whether or not this function is ever called.
+ *   - The array is part of the library image: a GPU holds the 32 MiB from the moment the library's
+ *     device code is loaded on it until the process exits.  With the CUDA runtime's default lazy module
+ *     loading that moment is the first call of this function on the device; with eager loading
+ *     (CUDA_MODULE_LOADING=EAGER) it is the first use of the library.  A caller inside a fixed memory
+ *     plan should therefore make one call at start-up, and must expect NOVA_ATTN_ERR_CUDA from it (code
+ *     in nova_attn_last_cuda_error) if the 32 MiB no longer fit on the device.
  *   - The call allocates nothing: no cudaMalloc, no cudaFree, no allocating library routine.
  *   - The first call on a device looks up the array's device address (one runtime query, cached per
  *     device).  Make that first call before starting any stream capture.
  *   - All calls on a device share the one array.  Each call clears the part it uses before use, so
  *     what an earlier call left behind is harmless, but two calls whose GPU work overlaps (different
  *     streams, or different host threads) race on it and corrupt each other's dQ.  Serialise them.
- *   - Arguments, validation, results and error codes are otherwise those of nova_attn_bwd.
+ *   - Arguments, validation, results and error codes are otherwise those of nova_attn_bwd, checked in
+ *     the same order: a NULL pointer, a bad shape, alignment or scale is reported as such even when the
+ *     problem is also too large for the array.
  */
 size_t nova_attn_static_scratch_bytes(void);
 int nova_attn_bwd_static_scratch(const void* Q, const void* K, const void* V, const void* O,

@@ -243,6 +243,21 @@ int check_shape(int B, int H, int T, int D) {
 }
 
 }  // namespace
+
+int record_cuda_error(int code) { return fail_cuda(code); }
+
+int validate_bwd_args(const void* Q, const void* K, const void* V, const void* dO, const float* LSE,
+                      const float* Delta, const void* dQ, const void* dK, const void* dV, int B, int H, int T, int D,
+                      float scale) {
+    if (!Q || !K || !V || !dO || !LSE || !Delta || !dQ || !dK || !dV) return NOVA_ATTN_ERR_NULL;
+    if (int rc = check_shape(B, H, T, D)) return rc;
+    if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(dO) || !aligned16(LSE) || !aligned16(Delta) ||
+        !aligned16(dQ) || !aligned16(dK) || !aligned16(dV))
+        return NOVA_ATTN_ERR_ALIGNMENT;
+    if (!std::isfinite(scale) || !(scale > 0.f)) return NOVA_ATTN_ERR_SCALE;
+    return NOVA_ATTN_OK;
+}
+
 }  // namespace nova
 
 using namespace nova;
@@ -344,12 +359,7 @@ int bwd_impl(const void* Q, const void* K, const void* V, const void* dO, const 
              const TensorStrides& sv, const TensorStrides& sdo, const TensorStrides& sdq, const TensorStrides& sdk,
              const TensorStrides& sdv, float scale, int causal, void* workspace, size_t workspace_bytes, void* stream,
              int steps) {
-    if (!Q || !K || !V || !dO || !LSE || !Delta || !dQ || !dK || !dV) return NOVA_ATTN_ERR_NULL;
-    if (int rc = check_shape(B, H, T, D)) return rc;
-    if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(dO) || !aligned16(LSE) || !aligned16(Delta) ||
-        !aligned16(dQ) || !aligned16(dK) || !aligned16(dV))
-        return NOVA_ATTN_ERR_ALIGNMENT;
-    if (!std::isfinite(scale) || !(scale > 0.f)) return NOVA_ATTN_ERR_SCALE;
+    if (int rc = validate_bwd_args(Q, K, V, dO, LSE, Delta, dQ, dK, dV, B, H, T, D, scale)) return rc;
     const size_t need = nova_attn_bwd_workspace_bytes(B, H, T, D);
     if (!workspace || workspace_bytes < need) return NOVA_ATTN_ERR_WORKSPACE;
     if (!aligned16(workspace)) return NOVA_ATTN_ERR_ALIGNMENT;
@@ -393,7 +403,7 @@ int nova_attn_bwd_steps(const void* Q, const void* K, const void* V, const void*
                         const float* Delta, void* dQ, void* dK, void* dV, int B, int H, int T, int D, float scale,
                         int causal, void* workspace, size_t workspace_bytes, void* stream, int steps) {
     (void)O;  // Delta already carries rowsum(dO * O)
-    if (int rc = check_shape(B, H, T, D)) return rc;
+    if (int rc = validate_bwd_args(Q, K, V, dO, LSE, Delta, dQ, dK, dV, B, H, T, D, scale)) return rc;
     const TensorStrides c = contiguous_strides(H, T, D);
     return bwd_impl(Q, K, V, dO, LSE, Delta, dQ, dK, dV, B, H, T, D, c, c, c, c, c, c, c, scale, causal, workspace,
                     workspace_bytes, stream, steps);
@@ -410,12 +420,7 @@ int nova_attn_bwd(const void* Q, const void* K, const void* V, const void* O, co
 int nova_attn_bwd_deterministic(const void* Q, const void* K, const void* V, const void* dO, const float* LSE,
                                 const float* Delta, void* dQ, void* dK, void* dV, int B, int H, int T, int D,
                                 float scale, int causal, void* stream) {
-    if (!Q || !K || !V || !dO || !LSE || !Delta || !dQ || !dK || !dV) return NOVA_ATTN_ERR_NULL;
-    if (int rc = check_shape(B, H, T, D)) return rc;
-    if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(dO) || !aligned16(LSE) || !aligned16(Delta) ||
-        !aligned16(dQ) || !aligned16(dK) || !aligned16(dV))
-        return NOVA_ATTN_ERR_ALIGNMENT;
-    if (!std::isfinite(scale) || !(scale > 0.f)) return NOVA_ATTN_ERR_SCALE;
+    if (int rc = validate_bwd_args(Q, K, V, dO, LSE, Delta, dQ, dK, dV, B, H, T, D, scale)) return rc;
     DeviceState* st = nullptr;
     if (int rc = device_state(&st)) return rc;
     const long long BH = static_cast<long long>(B) * H;

@@ -4,12 +4,15 @@
 // no allocator to ask: code running inside a framework's static memory plan, a plugin that is handed
 // only its input and output buffers, a real-time loop that must not call cudaMalloc after start-up.
 // For them the accumulator lives in the fixed array below, which is part of the library image: every
-// GPU that loads the library holds these 32 MiB until the process exits.
+// GPU on which the library's device code has been loaded holds these 32 MiB until the process exits.
+// (The CUDA runtime loads device code lazily by default: the array is then materialised by the first
+// call of this entry point on a device, not when the shared object is opened.)
 #include <cuda_runtime.h>
 
 #include <mutex>
 
 #include "../../include/nova_attn.h"
+#include "kernels.h"
 
 namespace {
 
@@ -51,12 +54,12 @@ size_t nova_attn_static_scratch_bytes(void) { return kStaticScratchBytes; }
 int nova_attn_bwd_static_scratch(const void* Q, const void* K, const void* V, const void* O, const void* dO,
                                  const float* LSE, const float* Delta, void* dQ, void* dK, void* dV, int B, int H,
                                  int T, int D, float scale, int causal, void* stream) {
-    const size_t need = nova_attn_bwd_workspace_bytes(B, H, T, D);
-    // need == 0 means an invalid shape: nova_attn_bwd below reports which argument is wrong.
-    if (need > kStaticScratchBytes) return NOVA_ATTN_ERR_WORKSPACE;
+    // Same order of checks as nova_attn_bwd: the arguments first, then the size of the accumulator.
+    if (int rc = nova::validate_bwd_args(Q, K, V, dO, LSE, Delta, dQ, dK, dV, B, H, T, D, scale)) return rc;
+    if (nova_attn_bwd_workspace_bytes(B, H, T, D) > kStaticScratchBytes) return NOVA_ATTN_ERR_WORKSPACE;
     float* scratch = nullptr;
     const cudaError_t e = static_scratch_address(&scratch);
-    if (e != cudaSuccess) return NOVA_ATTN_ERR_CUDA;
+    if (e != cudaSuccess) return nova::record_cuda_error(static_cast<int>(e));
     // Same kernels as nova_attn_bwd; it clears the part of the accumulator it uses on `stream` first,
     // so whatever the previous call left in the array does not matter.
     return nova_attn_bwd(Q, K, V, O, dO, LSE, Delta, dQ, dK, dV, B, H, T, D, scale, causal, scratch,

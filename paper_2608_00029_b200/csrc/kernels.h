@@ -25,6 +25,16 @@ struct TensorStrides {
     long long b, h, t;
 };
 
+// Records a CUDA error code for nova_attn_last_cuda_error() of the calling thread and returns
+// NOVA_ATTN_ERR_CUDA; for the entry points that live outside api.cu.
+int record_cuda_error(int code);
+
+// The argument checks every backward entry point makes before anything else (NULL pointers, shape, 16-byte
+// alignment of the tensors, scale); returns NOVA_ATTN_OK or the error nova_attn_bwd would report.
+int validate_bwd_args(const void* Q, const void* K, const void* V, const void* dO, const float* LSE,
+                      const float* Delta, const void* dQ, const void* dK, const void* dV, int B, int H, int T, int D,
+                      float scale);
+
 // Launches `kernel` allowing it to overlap the tail of the previous kernel in `stream` (programmatic
 // dependent launch); the kernel must call griddep_wait() before it touches global memory.
 template <typename... KArgs, typename... Args>

@@ -92,6 +92,28 @@ def test_deterministic_backward_validates_without_a_workspace(lib):
     assert d(*bad, 1, 1, 16, 64, 1.0, 1, None) == na.ERR_ALIGNMENT
 
 
+def test_static_scratch_backward_reports_argument_errors_before_the_size_limit(lib):
+    """A NULL pointer, an unsupported head dimension or a bad scale is reported as such even when the
+    problem would also be too large for the built-in array; only a valid, oversized problem gets the
+    workspace error.  None of these calls reaches the GPU."""
+    from paper_2608_00029_b200 import nova_attn as na
+    p = ctypes.c_void_p(0x1000)
+    s = lib.nova_attn_bwd_static_scratch
+    ptrs = [p] * 10
+    big = (3, 12, 4096)                                   # 9.4 Mi elements at D=64: more than the array holds
+    assert s(*ptrs, *big, 64, 1.0, 1, None) == na.ERR_WORKSPACE
+    assert s(*ptrs, *big, 96, 1.0, 1, None) == na.ERR_UNSUPPORTED
+    assert s(*ptrs, *big, 64, -1.0, 1, None) == na.ERR_SCALE
+    bad = list(ptrs)
+    bad[7] = None                                         # dQ
+    assert s(*bad, *big, 64, 1.0, 1, None) == na.ERR_NULL
+    bad[7] = ctypes.c_void_p(0x1004)
+    assert s(*bad, *big, 64, 1.0, 1, None) == na.ERR_ALIGNMENT
+    bad = list(ptrs)
+    bad[3] = None                                         # O is ignored, as in nova_attn_bwd
+    assert s(*bad, *big, 64, 1.0, 1, None) == na.ERR_WORKSPACE
+
+
 def test_strided_entry_points_validate_strides(lib):
     from paper_2608_00029_b200 import nova_attn as na
     p = ctypes.c_void_p(0x1000)
