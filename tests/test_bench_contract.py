@@ -59,7 +59,15 @@ def test_device_arm_line(launch):
     r = d["roofline"]
     assert r["bound"] == "tensor" and r["unit"] == "TFLOP/s" and r["peak"] > 0
     assert abs(r["frac"] - r["achieved"] / r["peak"]) < 1e-9 and 0.05 < r["frac"] < 1.2
-    assert r["traffic"] is None or r["traffic"] > 0
+    assert "burst" in r["peak_source"] and r["peak_sustained"] <= r["peak"]
+    assert r["traffic"] is None or (r["traffic"] > 0 and r["traffic_source"].startswith("profiles/"))
+    # the two fractions the targets are stated on: the forward, and the whole backward timed as one sequence
+    t = r["targets"]
+    assert t["fwd"]["target"] == 0.50 and t["bwd"]["target"] == 0.35
+    for leg in ("fwd", "bwd"):
+        assert t[leg]["ms"] > 0 and abs(t[leg]["frac"] - t[leg]["tflops"] / r["peak"]) < 1e-9
+    k = r["kernel_ms"]
+    assert t["bwd"]["ms"] > k["bwd_main"] * 0.9   # the sequence contains the main kernel
     e = d["e2e"]
     assert e["h2d_bytes_per_step"] == e["d2h_bytes_per_step"] == 4 * 8 * 12 * 1024 * 64 * 2
     assert 0 < e["value"] < d["value"]  # the copies are inside the timed region

@@ -23,49 +23,52 @@ def _harness():
     return gpu_harness
 
 
-def _sample_heads(cfg, n, seed=123):
-    rng = np.random.default_rng(seed)
-    all_heads = [(b, h) for b in range(cfg.B) for h in range(cfg.H)]
-    idx = rng.choice(len(all_heads), size=min(n, len(all_heads)), replace=False)
-    picked = {all_heads[i] for i in idx} | {all_heads[0], all_heads[-1]}
-    return sorted(picked)
+# name -> which preprocess produces Delta.  The GPU runs the full configuration and the oracle checks
+# EVERY head of it.  The peaked-softmax configuration is checked against the stated bounds with the exact
+# Delta; rowsum(dO * O) on it is covered by the next test.
+FIVE = [("tiny", False), ("gpt2_small", False), ("gpt2_small_large_batch", True), ("gpt2_medium", False),
+        ("long_context", False)]
 
 
-# name -> (number of heads the oracle checks (None = all), which preprocess produces Delta).
-# The GPU always runs the full configuration.  The peaked-softmax configuration is checked against
-# the stated bounds with the exact Delta; rowsum(dO * O) on it is covered by the next test.
-FIVE = [("tiny", None, False), ("gpt2_small", None, False), ("gpt2_small_large_batch", 24, True),
-        ("gpt2_medium", 24, False), ("long_context", 3, False)]
-
-
-@pytest.mark.parametrize("name,n_heads,exact_delta", FIVE)
-def test_five_configs_match_oracle(name, n_heads, exact_delta):
+@pytest.mark.parametrize("name,exact_delta", FIVE)
+def test_five_configs_match_oracle(name, exact_delta):
     h = _harness()
     cfg = W.CONFIGS[name]
     Q, K, V, dO = W.make_inputs(cfg)
     got = h.run_gpu(Q, K, V, dO, cfg.scale, cfg.causal, exact_delta=exact_delta)
-    heads = None if n_heads is None else _sample_heads(cfg, n_heads)
-    ref = h.run_oracle(Q, K, V, dO, cfg.scale, cfg.causal, heads)
-    errs = h.compare(h.select_heads(got, heads), ref, label=f"{name}: ", dO=ref["dO_in"])
+    ref = h.run_oracle(Q, K, V, dO, cfg.scale, cfg.causal)
+    errs = h.compare(h.select_heads(got, None), ref, label=f"{name}: ", dO=ref["dO_in"])
     print(name, {k: f"{v:.2e}" for k, v in errs.items()})
-    # properties that hold at any size, on ALL heads of the GPU result
+    # properties that hold at any size
     dK = W.widen(got["dK"])
     dK_abs = np.abs(dK).sum(2)
     assert (np.abs(dK.sum(2)) <= 2e-2 * dK_abs + 1e-3).all(), "sum_j dK_j should vanish per head"
     assert all(torch.isfinite(t.float()).all() for t in got.values())
 
 
+# Largest |err| / (2e-2 + 2e-2|ref|) over all 384 heads of the peaked configuration when Delta comes from
+# rowsum(dO * O), as measured on the GPU (see the figures printed by the test), plus a margin of 0.25.
+ROWSUM_ROUTE_FACTOR = 2.0
+
+
 def test_peaked_config_with_rowsum_delta():
-    """Peaked softmax with Delta = rowsum(dO * O): the bf16 rounding of O alone (see
-    test_delta_precision.py for the arithmetic, no GPU involved) pushes a few dQ/dK elements past
-    2e-2 + 2e-2|ref|, so this route is held to twice that bound and to the same relative RMS."""
+    """Peaked softmax through the three calls in their stated order (forward, rowsum preprocess, backward),
+    all heads.  The bf16 rounding of O alone (see test_delta_precision.py for the arithmetic, no GPU
+    involved) pushes some dQ/dK elements past 2e-2 + 2e-2|ref|: the test prints how many of which tensor
+    and by how much, and holds the route to the measured excess plus a margin, with the usual relative RMS."""
+    import tolerance as tol
     h = _harness()
     cfg = W.CONFIGS["gpt2_small_large_batch"]
     Q, K, V, dO = W.make_inputs(cfg)
     got = h.run_gpu(Q, K, V, dO, cfg.scale, True, exact_delta=False)
-    heads = _sample_heads(cfg, 24)
-    ref = h.run_oracle(Q, K, V, dO, cfg.scale, True, heads)
-    h.compare(h.select_heads(got, heads), ref, label="large_batch/rowsum: ", dO=ref["dO_in"], bwd_factor=2.0)
+    ref = h.run_oracle(Q, K, V, dO, cfg.scale, True)
+    sel = h.select_heads(got, None)
+    for name in ("dQ", "dK", "dV"):
+        n_bad, worst, n = tol.violation_stats(sel[name], ref[name], tol.BWD_ATOL, tol.BWD_RTOL)
+        per_head = (np.abs(sel[name] - ref[name]) > tol.BWD_ATOL + tol.BWD_RTOL * np.abs(ref[name])).any(axis=(2, 3))
+        print(f"large_batch/rowsum {name}: {n_bad} of {n} elements beyond 1x the bound, on {int(per_head.sum())} of "
+              f"{per_head.size} heads; largest error / bound = {worst:.3f}")
+    h.compare(sel, ref, label="large_batch/rowsum: ", dO=ref["dO_in"], bwd_factor=ROWSUM_ROUTE_FACTOR)
 
 
 def test_exact_delta_matches_jacobian_definition():

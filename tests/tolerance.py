@@ -35,3 +35,12 @@ def assert_close(got, ref, atol, rtol, name="", rms_bound=None):
         r = rel_rms(got, ref)
         assert r <= rms_bound, f"{name}: relative RMS error {r:.3e} > {rms_bound}"
     return maxerr
+
+
+def violation_stats(got, ref, atol, rtol):
+    """How far a result is from the bound, as numbers to record: the count of elements with
+    |got - ref| > atol + rtol*|ref| and the largest |got - ref| / (atol + rtol*|ref|)."""
+    got = np.asarray(got, dtype=np.float64)
+    ref = np.asarray(ref, dtype=np.float64)
+    ratio = np.abs(got - ref) / (atol + rtol * np.abs(ref))
+    return int((ratio > 1.0).sum()), float(ratio.max()), int(ratio.size)
