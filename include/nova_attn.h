@@ -233,6 +233,18 @@ const char* nova_attn_status_string(int status);
 int nova_attn_last_cuda_error(void);
 
 /*
+ * Test aid (the paper has no counterpart): lets a test make a bounded device-side wait run out without
+ * hanging or faulting anything.  Every spin-wait in the kernels gives up after a cycle limit, the kernel
+ * then drains its copies, frees its tensor memory and returns, and nova_attn_poll_device_status reports
+ * NOVA_ATTN_ERR_TIMEOUT.  `limit_cycles` sets that limit for kernels launched afterwards by this process
+ * (0 restores the default of 2^29 cycles, about a quarter of a second); it applies to nova_attn_fwd.
+ * `inject` = 1 makes that kernel's loader leave out the request for its first K tile, so that the wait for
+ * it expires; 0 is normal operation.  Returns NOVA_ATTN_ERR_SHAPE for a negative limit or an unknown
+ * `inject`.  Not for production use: outputs of a call made with inject = 1 are invalid by construction.
+ */
+int nova_attn_test_configure_waits(long long limit_cycles, int inject);
+
+/*
  * Synchronises `stream`, then reads and clears the device status word of the current device.
  * Returns NOVA_ATTN_OK, NOVA_ATTN_ERR_TIMEOUT (a kernel gave up on a bounded wait; its outputs are
  * invalid) or NOVA_ATTN_ERR_CUDA.

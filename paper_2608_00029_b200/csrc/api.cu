@@ -4,6 +4,7 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
+#include <atomic>
 #include <cmath>
 #include <cstdint>
 #include <cstring>
@@ -38,6 +39,10 @@ struct DeviceState {
 };
 std::mutex g_mutex;
 DeviceState g_devices[kMaxDevices];
+// Test aid (nova_attn_test_configure_waits): cycle limit of the device-side waits and the fault to inject.
+constexpr long long kDefaultWaitLimit = 1ll << 29;
+std::atomic<long long> g_wait_limit{kDefaultWaitLimit};
+std::atomic<int> g_inject{0};
 EncodeTiledFn g_encode = nullptr;
 
 // One-time set-up of the current device: capability check, opt-in shared memory sizes, address of
@@ -288,8 +293,10 @@ int nova_attn_fwd_strided(const void* Q, const void* K, const void* V, void* O, 
     if (int rc = get_bf16_map(V, s, sv, strided, &tmV, &ov)) return rc;
     if (int rc = get_bf16_map(O, s, so, strided, &tmO, &oo)) return rc;
     const uint32_t orders = oq | (ok << 4) | (ov << 8) | (oo << 12);
-    const cudaError_t e = launch_attn_fwd(tmQ, tmK, tmV, tmO, strided, orders, LSE, s, st->num_sms, st->dev_status,
-                                          static_cast<cudaStream_t>(stream));
+    const cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    const cudaError_t e = launch_attn_fwd(tmQ, tmK, tmV, tmO, strided, orders, LSE, s, st->num_sms,
+                                          g_wait_limit.load(std::memory_order_relaxed),
+                                          g_inject.load(std::memory_order_relaxed), st->dev_status, cs);
     return e == cudaSuccess ? NOVA_ATTN_OK : fail_cuda(e);
 }
 
@@ -479,6 +486,13 @@ const char* nova_attn_status_string(int status) {
 }
 
 int nova_attn_last_cuda_error(void) { return t_last_cuda_error; }
+
+int nova_attn_test_configure_waits(long long limit_cycles, int inject) {
+    if (limit_cycles < 0 || inject < 0 || inject > 1) return NOVA_ATTN_ERR_SHAPE;
+    g_wait_limit.store(limit_cycles == 0 ? kDefaultWaitLimit : limit_cycles, std::memory_order_relaxed);
+    g_inject.store(inject, std::memory_order_relaxed);
+    return NOVA_ATTN_OK;
+}
 
 int nova_attn_poll_device_status(void* stream) {
     DeviceState* st = nullptr;

@@ -86,6 +86,7 @@ struct BwdCfg {
     static constexpr bool kSeparateP = (D == 64);   // P^T in its own columns instead of over S^T
     static constexpr int kColP = kSeparateP ? 448 : 0;
     static constexpr int kPHalfStride = kSeparateP ? 32 : 64;  // column distance between the two query halves of P^T
+    static constexpr int kQPT = 64;            // queries per compute thread (128 / kQPT warpgroups of compute warps)
 };
 
 struct BwdBars {
@@ -392,14 +393,15 @@ __device__ __forceinline__ void bwd_rows(BwdBars* bars, float* row_buf, const fl
     }
 }
 
-// P phase for this thread's 64 queries: p = exp2(s*c - lse*log2e), packed to bf16 pairs.  `s_lse4`
-// holds -lse*log2e; the multiply-add runs on packed fp32 pairs.
+// P phase for this thread's N queries: p = exp2(s*c - lse*log2e), left in place of the scores as fp32
+// (the dS phase multiplies by the unrounded p: only what feeds a contraction is rounded to bf16, paper
+// Section 4.3).  `s_lse4` holds -lse*log2e; the multiply-add runs on packed fp32 pairs.
 // kMasked: the tile is the diagonal one and/or holds keys past the end of the sequence.
-template <bool kMasked>
-__device__ __forceinline__ void bwd_p_phase(const uint32_t (&sv)[64], const float4* s_lse4, float c, uint32_t (&pk)[32],
-                                            bool key_valid, bool diag, int r, int q_base) {
+template <bool kMasked, int N>
+__device__ __forceinline__ void bwd_p_phase(uint32_t (&sv)[N], const float4* s_lse4, float c, bool key_valid, bool diag,
+                                            int r, int q_base) {
 #pragma unroll
-    for (int g = 0; g < 16; ++g) {
+    for (int g = 0; g < N / 4; ++g) {
         const float4 l4 = s_lse4[g];
         const uint64_t c2 = f32x2_pack(c, c);
         float x0, x1, x2, x3;
@@ -416,8 +418,10 @@ __device__ __forceinline__ void bwd_p_phase(const uint32_t (&sv)[64], const floa
             if (!key_valid || (diag && r > q0 + 2)) p2 = 0.f;
             if (!key_valid || (diag && r > q0 + 3)) p3 = 0.f;
         }
-        pk[2 * g + 0] = pack_bf16x2(p0, p1);
-        pk[2 * g + 1] = pack_bf16x2(p2, p3);
+        sv[4 * g + 0] = __float_as_uint(p0);
+        sv[4 * g + 1] = __float_as_uint(p1);
+        sv[4 * g + 2] = __float_as_uint(p2);
+        sv[4 * g + 3] = __float_as_uint(p3);
     }
 }
 
@@ -440,22 +444,28 @@ __device__ __forceinline__ void bwd_store_dkv32(const uint32_t (&a)[32], const u
     }
 }
 
+// Compute warps.  A thread owns one key row and kQPT consecutive queries of the tile (64: two warpgroups;
+// 32: four), i.e. columns [kQPT*part, kQPT*(part+1)) of S^T and dP^T.
 template <int D, bool kCausal>
 __device__ __forceinline__ void bwd_compute(uint8_t* smem, BwdBars* bars, uint32_t tmem_base,
                                             __nv_bfloat16* __restrict__ dK, __nv_bfloat16* __restrict__ dV,
                                             const TensorStrides& sdk, const TensorStrides& sdv, int T, float scale,
                                             const WorkList& wl, int cwarp, int lane) {
     using Cfg = BwdCfg<D>;
+    constexpr int kQPT = Cfg::kQPT;
     volatile int* abort_flag = &bars->abort_flag;
     const uint32_t lane_base = 32u * (cwarp & 3);
-    const int half = cwarp >> 2;             // which 64 queries of the tile this thread covers
+    const int part = cwarp >> 2;             // which kQPT queries of the tile this thread covers
+    const int half = (part * kQPT) / 64;     // the 64-query half they lie in (a box of the dS^T staging buffer)
     const int r = lane_base + lane;          // local key row
     const float c = scale * kLog2e;
-    const uint32_t t_s = tmem_addr(tmem_base, lane_base, Cfg::kColS + 64 * half);
-    const uint32_t t_dp = tmem_addr(tmem_base, lane_base, Cfg::kColdP + 64 * half);
-    const uint32_t t_p = tmem_addr(tmem_base, lane_base, Cfg::kColP + Cfg::kPHalfStride * half);
+    const uint32_t t_s = tmem_addr(tmem_base, lane_base, Cfg::kColS + kQPT * part);
+    const uint32_t t_dp = tmem_addr(tmem_base, lane_base, Cfg::kColdP + kQPT * part);
+    // bf16 P^T: kQPT / 2 packed columns, in columns of their own or over this thread's own S^T columns
+    const uint32_t t_p = tmem_addr(tmem_base, lane_base, Cfg::kColP + (Cfg::kSeparateP ? kQPT / 2 : kQPT) * part);
     const float* row_buf = reinterpret_cast<const float*>(smem + Cfg::kOffRow);
     uint8_t* sdS_row = smem + Cfg::kOffdS + half * kHalfTileBytes + r * 128;
+    const int ch0 = ((part * kQPT) % 64) / 8;  // first 16-byte chunk of this thread's queries in the 128-byte row
     bool ok = true;
     int w = 0, g = 0;
 
@@ -469,89 +479,85 @@ __device__ __forceinline__ void bwd_compute(uint8_t* smem, BwdBars* bars, uint32
         for (int it = 0; it < n_it; ++it, ++g) {
             const int i = i0 + it;
             const int b = g & 1;
-            const float4* s_lse4 = reinterpret_cast<const float4*>(row_buf + b * 256 + 64 * half);
-            const float4* s_dl4 = reinterpret_cast<const float4*>(row_buf + b * 256 + 128 + 64 * half);
+            const float4* s_lse4 = reinterpret_cast<const float4*>(row_buf + b * 256 + kQPT * part);
+            const float4* s_dl4 = reinterpret_cast<const float4*>(row_buf + b * 256 + 128 + kQPT * part);
             ok = mbar_wait(&bars->row_full[b], (g >> 1) & 1, abort_flag);
             if (!ok) break;
             ok = mbar_wait(&bars->s_full, g & 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
 
-            // ---- P phase
-            uint32_t pk[32];
+            // ---- P phase: the scores become fp32 probabilities in place
+            uint32_t pf[kQPT];
+#pragma unroll
+            for (int x = 0; x < kQPT; x += 32) tmem_ld_x32(t_s + x, pf + x);
+            tmem_wait_ld();
             {
-                uint32_t sv[64];
-                tmem_ld_x32(t_s, sv);
-                tmem_ld_x32(t_s + 32, sv + 32);
-                tmem_wait_ld();
                 const bool diag = kCausal && (i == kt);
                 if (diag || !tile_keys_valid)
-                    bwd_p_phase<true>(sv, s_lse4, c, pk, key_valid, diag, r, 64 * half);
+                    bwd_p_phase<true, kQPT>(pf, s_lse4, c, key_valid, diag, r, kQPT * part);
                 else
-                    bwd_p_phase<false>(sv, s_lse4, c, pk, true, false, r, 64 * half);
+                    bwd_p_phase<false, kQPT>(pf, s_lse4, c, true, false, r, kQPT * part);
             }
-            // ---- dS phase: ds = p * (dp - delta); bf16 to TMEM (for dK) and to swizzled smem (for dQ).
-            // p is taken from the bf16 pairs already in registers.
-            // dP^T of this tile was queued after dQ of the previous one and the tensor pipe completes in
-            // order, so the dp_full wait also covers "the previous dQ has finished reading the dS staging
-            // buffer".  Where dP^T never waits for this tile's P^T (kEarlydP) its loads are issued before
-            // the P^T store is awaited, so the two TMEM round trips overlap.
+            // P^T as bf16 into TMEM for dV.  Where P^T has columns of its own (kEarlydP) the store must wait
+            // until dV of the previous tile has read them: dP^T of this tile was queued after that dV and the
+            // tensor pipe completes in order, so the dp_full wait covers it, and the first dP^T load is issued
+            // before the P^T store is awaited so that the two TMEM round trips overlap.
             constexpr bool kEarlydP = Cfg::kSeparateP && !Cfg::kdQAliased;
             static_assert(kEarlydP || !Cfg::kSeparateP, "P^T columns of their own need the dp_full wait below");
-            uint32_t dd[32];
-            {
-                uint32_t dv[64];
-                if (kEarlydP) {
-                    // dP^T of this tile was queued after dV of the previous one and the tensor pipe completes
-                    // in order, so this wait also covers "dV has finished reading the P^T columns".
-                    ok = mbar_wait(&bars->dp_full, g & 1, abort_flag);
-                    if (!ok) break;
-                    tc_fence_after();
-                    tmem_st_x32(t_p, pk);
-                    tmem_ld_x32(t_dp, dv);
-                    tmem_ld_x32(t_dp + 32, dv + 32);
-                    tmem_wait_st();
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&bars->p_ready);
-                } else {
-                    tmem_st_x32(t_p, pk);
-                    tmem_wait_st();
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&bars->p_ready);
-                    ok = mbar_wait(&bars->dp_full, g & 1, abort_flag);
-                    if (!ok) break;
-                    tc_fence_after();
-                    tmem_ld_x32(t_dp, dv);
-                    tmem_ld_x32(t_dp + 32, dv + 32);
-                }
-                tmem_wait_ld();
-#pragma unroll
-                for (int x = 0; x < 16; ++x) {
-                    const float4 d4 = s_dl4[x];
-                    const uint32_t pa = pk[2 * x], pb = pk[2 * x + 1];
-                    const float p0 = __uint_as_float(pa << 16), p1 = __uint_as_float(pa & 0xffff0000u);
-                    const float p2 = __uint_as_float(pb << 16), p3 = __uint_as_float(pb & 0xffff0000u);
-                    // d4 holds -delta: ds = p * (dp + (-delta)) on packed fp32 pairs
-                    float d0, d1, d2, d3;
-                    f32x2_unpack(f32x2_mul(f32x2_pack(p0, p1),
-                                           f32x2_add(f32x2_pack(__uint_as_float(dv[4 * x + 0]), __uint_as_float(dv[4 * x + 1])),
-                                                     f32x2_pack(d4.x, d4.y))), d0, d1);
-                    f32x2_unpack(f32x2_mul(f32x2_pack(p2, p3),
-                                           f32x2_add(f32x2_pack(__uint_as_float(dv[4 * x + 2]), __uint_as_float(dv[4 * x + 3])),
-                                                     f32x2_pack(d4.z, d4.w))), d2, d3);
-                    dd[2 * x + 0] = pack_bf16x2(d0, d1);
-                    dd[2 * x + 1] = pack_bf16x2(d2, d3);
-                }
+            if (kEarlydP) {
+                ok = mbar_wait(&bars->dp_full, g & 1, abort_flag);
+                if (!ok) break;
+                tc_fence_after();
             }
-            tmem_st_x32(t_dp, dd);
-            // dS^T row r, this half's 64 queries: eight 16-byte chunks of one 128-byte swizzled row.
-            if (!wl.no_dq) {
 #pragma unroll
-                for (int ch = 0; ch < 8; ++ch)
-                    *reinterpret_cast<uint4*>(sdS_row + ((ch ^ (r & 7)) << 4)) =
-                        make_uint4(dd[ch * 4 + 0], dd[ch * 4 + 1], dd[ch * 4 + 2], dd[ch * 4 + 3]);
+            for (int x = 0; x < kQPT; x += 32) {
+                uint32_t pk[16];
+#pragma unroll
+                for (int y = 0; y < 16; ++y)
+                    pk[y] = pack_bf16x2(__uint_as_float(pf[x + 2 * y]), __uint_as_float(pf[x + 2 * y + 1]));
+                tmem_st_x16(t_p + x / 2, pk);
+            }
+            uint32_t dv[16];
+            if (kEarlydP) tmem_ld_x16(t_dp, dv);
+            tmem_wait_st();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bars->p_ready);
+            if (!kEarlydP) {
+                ok = mbar_wait(&bars->dp_full, g & 1, abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+                tmem_ld_x16(t_dp, dv);
+            }
+            // ---- dS phase, 16 queries at a time: ds = p * (dp - delta) in fp32, rounded once to bf16, to TMEM
+            // (over this thread's own, already read dP^T columns) for dK and to swizzled smem for dQ.
+            // dP^T of this tile was queued after dQ of the previous one and the tensor pipe completes in order,
+            // so the dp_full wait also covers "the previous dQ has finished reading the dS staging buffer".
+#pragma unroll
+            for (int x = 0; x < kQPT; x += 16) {
+                tmem_wait_ld();
+                uint32_t dd[8];
+#pragma unroll
+                for (int y = 0; y < 4; ++y) {
+                    const float4 d4 = s_dl4[x / 4 + y];  // holds -delta
+                    float d0, d1, d2, d3;
+                    f32x2_unpack(f32x2_mul(f32x2_pack(__uint_as_float(pf[x + 4 * y + 0]), __uint_as_float(pf[x + 4 * y + 1])),
+                                           f32x2_add(f32x2_pack(__uint_as_float(dv[4 * y + 0]), __uint_as_float(dv[4 * y + 1])),
+                                                     f32x2_pack(d4.x, d4.y))), d0, d1);
+                    f32x2_unpack(f32x2_mul(f32x2_pack(__uint_as_float(pf[x + 4 * y + 2]), __uint_as_float(pf[x + 4 * y + 3])),
+                                           f32x2_add(f32x2_pack(__uint_as_float(dv[4 * y + 2]), __uint_as_float(dv[4 * y + 3])),
+                                                     f32x2_pack(d4.z, d4.w))), d2, d3);
+                    dd[2 * y + 0] = pack_bf16x2(d0, d1);
+                    dd[2 * y + 1] = pack_bf16x2(d2, d3);
+                }
+                if (x + 16 < kQPT) tmem_ld_x16(t_dp + x + 16, dv);  // all of dv has been consumed above
+                tmem_st_x8(t_dp + x / 2, dd);
+                if (!wl.no_dq) {  // dS^T row r: two 16-byte chunks of one 128-byte swizzled row
+                    const int ch = ch0 + x / 8;
+                    *reinterpret_cast<uint4*>(sdS_row + (((ch + 0) ^ (r & 7)) << 4)) = make_uint4(dd[0], dd[1], dd[2], dd[3]);
+                    *reinterpret_cast<uint4*>(sdS_row + (((ch + 1) ^ (r & 7)) << 4)) = make_uint4(dd[4], dd[5], dd[6], dd[7]);
+                }
             }
             tmem_wait_st();
             fence_proxy_async_smem();
@@ -690,19 +696,23 @@ __device__ __forceinline__ void bwd_dq_tma(uint8_t* smem, BwdBars* bars, uint32_
         if (!ok) break;
         tc_fence_after();
         uint32_t pv[32], pk[32];
-        {
-            uint32_t a[64];
-            tmem_ld_x32(t_dv, a);
-            tmem_ld_x32(t_dv + 32, a + 32);
+#pragma unroll
+        for (int cb = 0; cb < 64; cb += 32) {  // 32 accumulator columns at a time keeps the register count down
+            uint32_t a[32];
+            tmem_ld_x32(t_dv + cb, a);
             tmem_wait_ld();
 #pragma unroll
-            for (int x = 0; x < 32; ++x) pv[x] = pack_bf16x2(__uint_as_float(a[2 * x]), __uint_as_float(a[2 * x + 1]));
-            tmem_ld_x32(t_dk, a);
-            tmem_ld_x32(t_dk + 32, a + 32);
+            for (int x = 0; x < 16; ++x)
+                pv[cb / 2 + x] = pack_bf16x2(__uint_as_float(a[2 * x]), __uint_as_float(a[2 * x + 1]));
+        }
+#pragma unroll
+        for (int cb = 0; cb < 64; cb += 32) {
+            uint32_t a[32];
+            tmem_ld_x32(t_dk + cb, a);
             tmem_wait_ld();
 #pragma unroll
-            for (int x = 0; x < 32; ++x)
-                pk[x] = pack_bf16x2(__uint_as_float(a[2 * x]) * scale, __uint_as_float(a[2 * x + 1]) * scale);
+            for (int x = 0; x < 16; ++x)
+                pk[cb / 2 + x] = pack_bf16x2(__uint_as_float(a[2 * x]) * scale, __uint_as_float(a[2 * x + 1]) * scale);
         }
         tc_fence_before();
         __syncwarp();

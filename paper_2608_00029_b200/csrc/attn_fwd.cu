@@ -87,7 +87,7 @@ struct FwdWork {
 template <int D, bool kStrided>
 __device__ __forceinline__ void fwd_producer(const CUtensorMap* tmQ, const CUtensorMap* tmK,
                                              const CUtensorMap* tmV, uint8_t* smem, FwdBars* bars,
-                                             const FwdWork& wk) {
+                                             const FwdWork& wk, long long limit, int inject) {
     using Cfg = FwdCfg<D>;
     volatile int* abort_flag = &bars->abort_flag;
     int armed_q[2] = {-1, -1}, armed_k[2] = {-1, -1}, armed_v[2] = {-1, -1};
@@ -99,7 +99,7 @@ __device__ __forceinline__ void fwd_producer(const CUtensorMap* tmQ, const CUten
         const int head = kStrided ? bh % wk.H : 0, batch = kStrided ? bh / wk.H : 0;
         const int qs = w % Cfg::kQStages;
         const uint32_t qph = (w / Cfg::kQStages) & 1;
-        ok = mbar_wait(&bars->q_empty[qs], qph ^ 1, abort_flag);
+        ok = mbar_wait(&bars->q_empty[qs], qph ^ 1, abort_flag, limit);
         if (!ok) break;
         mbar_expect_tx(&bars->q_full[qs], 2 * Cfg::kTileBytes);  // rows past T arrive as zeros
         armed_q[qs] = qph;
@@ -113,15 +113,20 @@ __device__ __forceinline__ void fwd_producer(const CUtensorMap* tmQ, const CUten
         for (int j = 0; j < n; ++j, ++g) {
             const int st = g & 1;
             const uint32_t ph = (g >> 1) & 1;
-            ok = mbar_wait(&bars->k_empty[st], ph ^ 1, abort_flag);
+            ok = mbar_wait(&bars->k_empty[st], ph ^ 1, abort_flag, limit);
             if (!ok) break;
-            mbar_expect_tx(&bars->k_full[st], Cfg::kTileBytes);
-            armed_k[st] = ph;
+            // `inject` (a test aid, 0 in normal use): the very first K tile is never requested, so the wait for
+            // it runs out and the kernel leaves through its time-out path
+            if (!(inject == 1 && g == 0)) {
+                mbar_expect_tx(&bars->k_full[st], Cfg::kTileBytes);
+                armed_k[st] = ph;
 #pragma unroll
-            for (int h = 0; h < Cfg::kHalves; ++h)
-                tma_load_tile<kStrided>(smem + Cfg::kOffK + st * Cfg::kTileBytes + h * kHalfTileBytes, tmK, &bars->k_full[st],
-                              (wk.orders >> 4) & 15, h * kBoxCols, j * kBlockK, head, batch, bh);
-            ok = mbar_wait(&bars->v_empty[st], ph ^ 1, abort_flag);
+                for (int h = 0; h < Cfg::kHalves; ++h)
+                    tma_load_tile<kStrided>(smem + Cfg::kOffK + st * Cfg::kTileBytes + h * kHalfTileBytes, tmK,
+                                            &bars->k_full[st], (wk.orders >> 4) & 15, h * kBoxCols, j * kBlockK, head,
+                                            batch, bh);
+            }
+            ok = mbar_wait(&bars->v_empty[st], ph ^ 1, abort_flag, limit);
             if (!ok) break;
             mbar_expect_tx(&bars->v_full[st], Cfg::kTileBytes);
             armed_v[st] = ph;
@@ -144,7 +149,8 @@ __device__ __forceinline__ void fwd_producer(const CUtensorMap* tmQ, const CUten
 }
 
 template <int D>
-__device__ __forceinline__ void fwd_mma(uint8_t* smem, FwdBars* bars, uint32_t tmem_base, const FwdWork& wk) {
+__device__ __forceinline__ void fwd_mma(uint8_t* smem, FwdBars* bars, uint32_t tmem_base, const FwdWork& wk,
+                                        long long limit) {
     using Cfg = FwdCfg<D>;
     volatile int* abort_flag = &bars->abort_flag;
     constexpr uint32_t kIdescQK = umma_idesc_bf16(128, 128, 0, 0);
@@ -172,7 +178,7 @@ __device__ __forceinline__ void fwd_mma(uint8_t* smem, FwdBars* bars, uint32_t t
         const uint32_t t_s = tmem_base + Cfg::kColS + 128 * t;
         const uint32_t b = k_k[gk & 1];
         if (Cfg::kSepP && cq[t] > 0) {  // the softmax warps must have read the previous S_t
-            ok = mbar_wait(&bars->s_free[t], (cq[t] - 1) & 1, abort_flag);
+            ok = mbar_wait(&bars->s_free[t], (cq[t] - 1) & 1, abort_flag, limit);
             if (!ok) return;
             tc_fence_after();
         }
@@ -198,8 +204,8 @@ __device__ __forceinline__ void fwd_mma(uint8_t* smem, FwdBars* bars, uint32_t t
 #pragma unroll
         for (int t = 0; t < 2; ++t)
             q_k[t] = umma_desc_lo(smem_u32(smem + Cfg::kOffQ + (qs * 2 + t) * Cfg::kTileBytes), 16);
-        ok = mbar_wait(&bars->q_full[qs], (w / Cfg::kQStages) & 1, abort_flag);
-        if (ok) ok = mbar_wait(&bars->k_full[g & 1], (g >> 1) & 1, abort_flag);
+        ok = mbar_wait(&bars->q_full[qs], (w / Cfg::kQStages) & 1, abort_flag, limit);
+        if (ok) ok = mbar_wait(&bars->k_full[g & 1], (g >> 1) & 1, abort_flag, limit);
         if (!ok) break;
         tc_fence_after();
         // P over S: the S columns of both tiles are free, their last P was consumed by a P V queued
@@ -215,7 +221,7 @@ __device__ __forceinline__ void fwd_mma(uint8_t* smem, FwdBars* bars, uint32_t t
             if (Cfg::kSepP && j + 1 < n) {
                 // Both Q K^T of the next key tile go first: S_t was released right after the softmax
                 // warps loaded it, long before their P is ready.
-                ok = mbar_wait(&bars->k_full[st ^ 1], ((g + 1) >> 1) & 1, abort_flag);
+                ok = mbar_wait(&bars->k_full[st ^ 1], ((g + 1) >> 1) & 1, abort_flag, limit);
                 if (!ok) break;
                 tc_fence_after();
 #pragma unroll
@@ -228,14 +234,14 @@ __device__ __forceinline__ void fwd_mma(uint8_t* smem, FwdBars* bars, uint32_t t
                 if (j >= n_t[t]) continue;
                 const uint32_t t_s = tmem_base + Cfg::kColP + Cfg::kStrideP * t;
                 const uint32_t t_o = tmem_base + Cfg::kColO + D * t;
-                ok = mbar_wait(&bars->p_ready[t], c[t] & 1, abort_flag);
+                ok = mbar_wait(&bars->p_ready[t], c[t] & 1, abort_flag, limit);
                 if (!ok) break;
                 if (j == 0) {
-                    ok = mbar_wait(&bars->v_full[st], (g >> 1) & 1, abort_flag);
+                    ok = mbar_wait(&bars->v_full[st], (g >> 1) & 1, abort_flag, limit);
                     // the previous item's O_t must have been read out of TMEM before it is overwritten
-                    if (ok && wt[t] > 0) ok = mbar_wait(&bars->o_free[t], (wt[t] - 1) & 1, abort_flag);
+                    if (ok && wt[t] > 0) ok = mbar_wait(&bars->o_free[t], (wt[t] - 1) & 1, abort_flag, limit);
                 } else if (t == 0 || j >= n_t[0]) {
-                    ok = mbar_wait(&bars->v_full[st], (g >> 1) & 1, abort_flag);
+                    ok = mbar_wait(&bars->v_full[st], (g >> 1) & 1, abort_flag, limit);
                 }
                 if (!ok) break;
                 tc_fence_after();
@@ -252,7 +258,7 @@ __device__ __forceinline__ void fwd_mma(uint8_t* smem, FwdBars* bars, uint32_t t
                 ++c[t];
                 if (!Cfg::kSepP && j + 1 < n_t[t]) {  // the S_t columns are free again once this P V has run
                     if (!next_k_ready) {
-                        ok = mbar_wait(&bars->k_full[st ^ 1], ((g + 1) >> 1) & 1, abort_flag);
+                        ok = mbar_wait(&bars->k_full[st ^ 1], ((g + 1) >> 1) & 1, abort_flag, limit);
                         if (!ok) break;
                         tc_fence_after();
                         next_k_ready = true;
@@ -283,7 +289,7 @@ __device__ __forceinline__ void fwd_mma(uint8_t* smem, FwdBars* bars, uint32_t t
 template <int D, bool kCausal, bool kStrided>
 __device__ __forceinline__ void fwd_softmax(uint8_t* smem, FwdBars* bars, uint32_t tmem_base, const CUtensorMap* tmO,
                                             float* __restrict__ LSE, float scale, const FwdWork& wk, int t, int swarp,
-                                            int lane) {
+                                            int lane, long long limit) {
     using Cfg = FwdCfg<D>;
     volatile int* abort_flag = &bars->abort_flag;
     const uint32_t lane_base = 32u * (swarp & 3);
@@ -310,7 +316,7 @@ __device__ __forceinline__ void fwd_softmax(uint8_t* smem, FwdBars* bars, uint32
             // has been filled, so that this warpgroup never runs ahead of the ring.
             bool leader_ok = true;
             if (leader) {
-                leader_ok = mbar_wait(&bars->q_full[qs], (w / Cfg::kQStages) & 1, abort_flag);
+                leader_ok = mbar_wait(&bars->q_full[qs], (w / Cfg::kQStages) & 1, abort_flag, limit);
                 if (leader_ok) mbar_arrive(&bars->q_empty[qs]);
             }
             ok = __all_sync(0xffffffffu, leader_ok);
@@ -321,7 +327,7 @@ __device__ __forceinline__ void fwd_softmax(uint8_t* smem, FwdBars* bars, uint32
         float l = 0.f;
 
         for (int j = 0; j < n_kv; ++j, ++cnt) {
-            ok = mbar_wait(&bars->s_full[t], cnt & 1, abort_flag);
+            ok = mbar_wait(&bars->s_full[t], cnt & 1, abort_flag, limit);
             if (!ok) break;
             tc_fence_after();
             uint32_t sr[128];
@@ -367,7 +373,7 @@ __device__ __forceinline__ void fwd_softmax(uint8_t* smem, FwdBars* bars, uint32
                     const float f = ex2_approx((m_ref - m_new) * c);  // 1 for rows whose maximum did not move
                     m_ref = m_new;
                     l *= f;
-                    ok = mbar_wait(&bars->pv_done[t], (cnt - 1) & 1, abort_flag);
+                    ok = mbar_wait(&bars->pv_done[t], (cnt - 1) & 1, abort_flag, limit);
                     if (!ok) break;
                     tc_fence_after();
                     #pragma unroll 1
@@ -386,7 +392,7 @@ __device__ __forceinline__ void fwd_softmax(uint8_t* smem, FwdBars* bars, uint32
             const uint64_t nmc2 = f32x2_pack(-m_ref * c, -m_ref * c);
             uint64_t acc0 = 0, acc1 = 0;  // two pairs of partial sums
             if (Cfg::kSepP && j > 0) {  // the previous P_t must have been consumed (long since, as a rule)
-                ok = mbar_wait(&bars->pv_done[t], (cnt - 1) & 1, abort_flag);
+                ok = mbar_wait(&bars->pv_done[t], (cnt - 1) & 1, abort_flag, limit);
                 if (!ok) break;
                 tc_fence_after();
             }
@@ -425,7 +431,7 @@ __device__ __forceinline__ void fwd_softmax(uint8_t* smem, FwdBars* bars, uint32
 
         // ---- end of the item: O_t / l as bf16 into this tile's Q buffer (no longer read: every
         // Q K^T of the tile completed before its last P V), then TMA stores; LSE straight to global.
-        ok = mbar_wait(&bars->pv_done[t], (cnt - 1) & 1, abort_flag);
+        ok = mbar_wait(&bars->pv_done[t], (cnt - 1) & 1, abort_flag, limit);
         if (!ok) break;
         tc_fence_after();
         const float inv_l = 1.0f / l;
@@ -456,7 +462,7 @@ __device__ __forceinline__ void fwd_softmax(uint8_t* smem, FwdBars* bars, uint32
         if (row < T) LSE[static_cast<size_t>(bh) * T + row] = m_ref * scale + logf(l);
         bool leader_ok = true;
         if (leader) {
-            leader_ok = mbar_wait(&bars->o_staged[t], wt & 1, abort_flag);
+            leader_ok = mbar_wait(&bars->o_staged[t], wt & 1, abort_flag, limit);
             if (leader_ok) {
 #pragma unroll
                 for (int h = 0; h < Cfg::kHalves; ++h)
@@ -481,7 +487,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1)
 attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
                 float* __restrict__ LSE, int T, int BH, int H, uint32_t orders, int n_blocks, float scale,
-                int* __restrict__ dev_status) {
+                long long limit, int inject, int* __restrict__ dev_status) {
     using Cfg = FwdCfg<D>;
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -538,12 +544,12 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     griddep_wait();  // everything above overlaps the previous kernel of the stream
 
     if (warp == 0) {
-        if (lane == 0) fwd_producer<D, kStrided>(&tmQ, &tmK, &tmV, smem, bars, wk);
+        if (lane == 0) fwd_producer<D, kStrided>(&tmQ, &tmK, &tmV, smem, bars, wk, limit, inject);
     } else if (warp == 1) {
-        fwd_mma<D>(smem, bars, tmem_base, wk);
+        fwd_mma<D>(smem, bars, tmem_base, wk, limit);
     } else if (warp >= 4) {
         const int t = (warp - 4) >> 2;
-        fwd_softmax<D, kCausal, kStrided>(smem, bars, tmem_base, &tmO, LSE, scale, wk, t, (warp - 4) & 3, lane);
+        fwd_softmax<D, kCausal, kStrided>(smem, bars, tmem_base, &tmO, LSE, scale, wk, t, (warp - 4) & 3, lane, limit);
     }
 
     tc_fence_before();
@@ -555,16 +561,16 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 template <int D, bool kCausal>
 cudaError_t launch_one(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV,
                        const CUtensorMap& tmO, bool strided, uint32_t orders, float* LSE, const AttnShape& s,
-                       int num_sms, int* dev_status, cudaStream_t stream) {
+                       int num_sms, long long wait_limit, int inject, int* dev_status, cudaStream_t stream) {
     const int n_blocks = (s.T + kBlockRows - 1) / kBlockRows;
     const int BH = s.B * s.H;
     const long long n_items = static_cast<long long>(n_blocks) * BH;
     const dim3 grid(static_cast<unsigned>(n_items < num_sms ? n_items : num_sms));  // one persistent CTA per SM
     if (strided)
         return launch_overlapped(attn_fwd_kernel<D, kCausal, true>, grid, dim3(kFwdThreads), FwdCfg<D>::kSmemBytes,
-                                 stream, tmQ, tmK, tmV, tmO, LSE, s.T, BH, s.H, orders, n_blocks, s.scale, dev_status);
+                                 stream, tmQ, tmK, tmV, tmO, LSE, s.T, BH, s.H, orders, n_blocks, s.scale, wait_limit, inject, dev_status);
     return launch_overlapped(attn_fwd_kernel<D, kCausal, false>, grid, dim3(kFwdThreads), FwdCfg<D>::kSmemBytes, stream,
-                             tmQ, tmK, tmV, tmO, LSE, s.T, BH, s.H, orders, n_blocks, s.scale, dev_status);
+                             tmQ, tmK, tmV, tmO, LSE, s.T, BH, s.H, orders, n_blocks, s.scale, wait_limit, inject, dev_status);
 }
 
 template <int D, bool kCausal, bool kStrided>
@@ -587,13 +593,13 @@ cudaError_t configure_attn_fwd() {
 
 cudaError_t launch_attn_fwd(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV,
                             const CUtensorMap& tmO, bool strided, uint32_t orders, float* LSE, const AttnShape& s,
-                            int num_sms, int* dev_status, cudaStream_t stream) {
+                            int num_sms, long long wait_limit, int inject, int* dev_status, cudaStream_t stream) {
     if (s.D == 64) {
-        return s.causal ? launch_one<64, true>(tmQ, tmK, tmV, tmO, strided, orders, LSE, s, num_sms, dev_status, stream)
-                        : launch_one<64, false>(tmQ, tmK, tmV, tmO, strided, orders, LSE, s, num_sms, dev_status, stream);
+        return s.causal ? launch_one<64, true>(tmQ, tmK, tmV, tmO, strided, orders, LSE, s, num_sms, wait_limit, inject, dev_status, stream)
+                        : launch_one<64, false>(tmQ, tmK, tmV, tmO, strided, orders, LSE, s, num_sms, wait_limit, inject, dev_status, stream);
     }
-    return s.causal ? launch_one<128, true>(tmQ, tmK, tmV, tmO, strided, orders, LSE, s, num_sms, dev_status, stream)
-                    : launch_one<128, false>(tmQ, tmK, tmV, tmO, strided, orders, LSE, s, num_sms, dev_status, stream);
+    return s.causal ? launch_one<128, true>(tmQ, tmK, tmV, tmO, strided, orders, LSE, s, num_sms, wait_limit, inject, dev_status, stream)
+                    : launch_one<128, false>(tmQ, tmK, tmV, tmO, strided, orders, LSE, s, num_sms, wait_limit, inject, dev_status, stream);
 }
 
 }  // namespace nova

@@ -58,10 +58,11 @@ inline cudaError_t launch_overlapped(void (*kernel)(KArgs...), dim3 grid, dim3 b
 // the maps are 4-D [D, x, y, z] with token / head / batch in order of increasing stride, and `orders`
 // holds, four bits per tensor in the order Q, K, V, O, which of the three sits where (see
 // tma_load_tile).  `tmO` describes the output and is used for TMA stores.  Persistent: launches at most
-// `num_sms` CTAs.
+// `num_sms` CTAs.  `wait_limit`: cycle limit of every device-side wait; `inject`: test aid, 1 makes the
+// loader leave out its first K-tile request so that a wait runs out (0 in normal use).
 cudaError_t launch_attn_fwd(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV,
                             const CUtensorMap& tmO, bool strided, uint32_t orders, float* LSE, const AttnShape& s,
-                            int num_sms, int* dev_status, cudaStream_t stream);
+                            int num_sms, long long wait_limit, int inject, int* dev_status, cudaStream_t stream);
 cudaError_t configure_attn_fwd();
 
 cudaError_t launch_attn_bwd_preprocess(const __nv_bfloat16* O, const __nv_bfloat16* dO, float* Delta,

@@ -75,10 +75,11 @@ __device__ __forceinline__ bool mbar_try_wait_suspend(uint64_t* bar, uint32_t pa
     return ok != 0;
 }
 
-// Bounded wait.  Returns false if the phase did not complete within kWaitLimitCycles or if another
+// Bounded wait.  Returns false if the phase did not complete within `limit` cycles or if another
 // thread of the CTA already gave up (*abort_flag != 0); the caller then leaves through the common
 // exit path.  `abort_flag` lives in shared memory.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                          long long limit = kWaitLimitCycles) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     for (;;) {
@@ -86,7 +87,25 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
         for (int i = 0; i < 8; ++i)
             if (mbar_try_wait_suspend(bar, parity, 20000u)) return true;
         if (*abort_flag != 0) return false;
-        if (clock64() - t0 > kWaitLimitCycles) {
+        if (clock64() - t0 > limit) {
+            *abort_flag = 1;
+            return false;
+        }
+    }
+}
+
+// The same bounded wait for a role that can afford to notice the completion up to `sleep_ns` late (a
+// loader running stages ahead): it sleeps between two tests instead of polling, so that it takes next to no
+// issue slots from the warps that share its scheduler.
+__device__ __forceinline__ bool mbar_wait_relaxed(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                                  long long limit, unsigned sleep_ns) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (;;) {
+        __nanosleep(sleep_ns);
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag != 0) return false;
+        if (clock64() - t0 > limit) {
             *abort_flag = 1;
             return false;
         }
@@ -306,6 +325,11 @@ __device__ __forceinline__ void tmem_ld_x16(uint32_t taddr, uint32_t* r) {
         : NOVA_R4(r, 0), NOVA_R4(r, 4), NOVA_R4(r, 8), NOVA_R4(r, 12)
         : "r"(taddr)
         : "memory");
+}
+__device__ __forceinline__ void tmem_st_x8(uint32_t taddr, const uint32_t* r) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%8], {%0, %1, %2, %3, %4, %5, %6, %7};" ::NOVA_W4(r, 0),
+                 NOVA_W4(r, 4), "r"(taddr)
+                 : "memory");
 }
 __device__ __forceinline__ void tmem_st_x32(uint32_t taddr, const uint32_t* r) {
     asm volatile(

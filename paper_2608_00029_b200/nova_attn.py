@@ -75,6 +75,8 @@ def load():
     lib.nova_attn_bwd_static_scratch.restype = i
     lib.nova_attn_static_scratch_bytes.argtypes = []
     lib.nova_attn_static_scratch_bytes.restype = sz
+    lib.nova_attn_test_configure_waits.argtypes = [ctypes.c_longlong, i]
+    lib.nova_attn_test_configure_waits.restype = i
     _lib = lib
     return lib
 
@@ -207,6 +209,14 @@ def nova_attn_bwd_static_scratch(Q, K, V, O, dO, LSE, Delta, dQ, dK, dV, scale: 
                                              int(bool(causal)), _stream_ptr(stream))
     if rc != OK:
         raise NovaAttnError(rc, "nova_attn_bwd_static_scratch")
+
+
+def nova_attn_test_configure_waits(limit_cycles: int = 0, inject: int = 0) -> None:
+    """Test aid: cycle limit of the device-side waits of kernels launched from now on (0 = default) and,
+    with inject=1, a forward whose loader leaves out one K-tile request so that a wait runs out."""
+    rc = load().nova_attn_test_configure_waits(int(limit_cycles), int(inject))
+    if rc != OK:
+        raise NovaAttnError(rc, "nova_attn_test_configure_waits")
 
 
 def nova_attn_poll_device_status(stream=None) -> int:

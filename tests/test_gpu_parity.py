@@ -47,8 +47,11 @@ def test_five_configs_match_oracle(name, exact_delta):
 
 
 # Largest |err| / (2e-2 + 2e-2|ref|) over all 384 heads of the peaked configuration when Delta comes from
-# rowsum(dO * O), as measured on the GPU (see the figures printed by the test), plus a margin of 0.25.
-ROWSUM_ROUTE_FACTOR = 2.0
+# rowsum(dO * O).  Measured on the GPU (B200): dQ 2.136 (1516 of 25.2 M elements beyond 1x, on 312 heads),
+# dK 2.165 (748 elements, 274 heads), dV 0.724 (none).  A float64 emulation of all 384 heads in which only O
+# (inside Delta), dS and the results are rounded to bf16 gives 2.05 / 2.02 (863 / 320 elements): the excess
+# belongs to the route, not to the kernels.  The bound is the measured figure plus a margin of about 0.25.
+ROWSUM_ROUTE_FACTOR = 2.4
 
 
 def test_peaked_config_with_rowsum_delta():
@@ -158,15 +161,15 @@ def test_benchmark_grid_shapes(B, H, T, D, causal, n_heads):
 
 def test_peaked_softmax_large_scores():
     """Scores ~ N(0, 16^2) (Q, K ~ 4 N(0,1)): exercises the running-max rescale and the exp range far
-    beyond the five configurations.  |K| and |dS| are 4x and ~10x larger than there, and dQ, dK are sums
-    of a few large bf16-rounded terms dS*K, so the gradients are held to three times the usual bound
-    (forward results to the usual one)."""
+    beyond the five configurations, with the exact Delta, at the stated bounds.  (dS is formed from the
+    unrounded probabilities: with P rounded to bf16 before that product the same case needs about twice
+    the gradient bound, as a float64 emulation with exactly those roundings shows.)"""
     h = _harness()
     cfg = W.AttnConfig("peaked", B=1, H=4, T=512, D=64, seed=77, qk_factor=4.0)
     Q, K, V, dO = W.make_inputs(cfg)
     got = h.run_gpu(Q, K, V, dO, cfg.scale, True, exact_delta=True)
     ref = h.run_oracle(Q, K, V, dO, cfg.scale, True)
-    h.compare(h.select_heads(got, None), ref, label="peaked: ", dO=ref["dO_in"], bwd_factor=3.0)
+    h.compare(h.select_heads(got, None), ref, label="peaked: ", dO=ref["dO_in"])
 
 
 def test_increasing_scores_force_rescales():
