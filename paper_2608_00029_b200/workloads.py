@@ -59,6 +59,48 @@ CONFIGS = {
 CONFIG_ORDER = ["tiny", "gpt2_small", "gpt2_small_large_batch", "gpt2_medium", "long_context"]
 
 
+@dataclasses.dataclass(frozen=True)
+class LmHeadConfig:
+    """Loss head of a language model: hidden states X [M, K] against the vocabulary matrix W [N, K]."""
+    name: str
+    M: int
+    N: int
+    K: int
+    seed: int
+    x_factor: float = 1.0      # hidden states after the final normalisation: unit scale
+    w_factor: float = 0.02     # GPT-2's initialisation scale of the (tied) embedding matrix
+    ignored_every: int = 0     # every so-many-th row gets the target -1 (a position without a label); 0 = none
+
+    @property
+    def flops(self) -> float:
+        """FLOPs of the projection: 2*M*N*K."""
+        return 2.0 * self.M * self.N * self.K
+
+    def replace(self, **kw) -> "LmHeadConfig":
+        return dataclasses.replace(self, **kw)
+
+
+# The paper measures its fused loss head on 8192 x 768 x 50304 (8 sequences of 1024 tokens, GPT-2-small width,
+# vocabulary padded to 50304: Section 6.1, "Fused Loss Head").
+LM_HEAD_CONFIGS = {
+    "lm_head_tiny": LmHeadConfig("lm_head_tiny", M=200, N=1000, K=64, seed=10, ignored_every=7),
+    "lm_head_gpt2": LmHeadConfig("lm_head_gpt2", M=8192, N=50304, K=768, seed=11),
+}
+
+
+def make_lmhead_inputs(cfg: LmHeadConfig, seed: int | None = None):
+    """Return (X bf16 [M,K], W bf16 [N,K], targets int32 [M]) as CPU tensors: X, W iid normal times their
+    factors, rounded to bf16; targets uniform over the vocabulary."""
+    g = torch.Generator(device="cpu")
+    g.manual_seed(cfg.seed if seed is None else seed)
+    X = (torch.randn((cfg.M, cfg.K), dtype=torch.float32, generator=g) * cfg.x_factor).to(torch.bfloat16)
+    W = (torch.randn((cfg.N, cfg.K), dtype=torch.float32, generator=g) * cfg.w_factor).to(torch.bfloat16)
+    t = torch.randint(0, cfg.N, (cfg.M,), generator=g, dtype=torch.int64).to(torch.int32)
+    if cfg.ignored_every > 0:
+        t[:: cfg.ignored_every] = -1
+    return X, W, t
+
+
 def make_inputs(cfg: AttnConfig, seed: int | None = None):
     """Return (Q, K, V, dO) as CPU bf16 tensors of shape [B,H,T,D]."""
     g = torch.Generator(device="cpu")
