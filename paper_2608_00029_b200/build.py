@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libnova_attn.so")
 SOURCES = ["api.cu", "attn_fwd.cu", "attn_bwd.cu", "attn_bwd_pre.cu", "attn_delta.cu", "attn_dq.cu",
-           "attn_bwd_static.cu"]
+           "attn_bwd_static.cu", "lmhead.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-shared", "-cudart", "shared"]
 
@@ -24,6 +24,7 @@ def _stale() -> bool:
     t = os.path.getmtime(LIB)
     deps = _sources() + [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".h", ".cuh"))]
     deps.append(os.path.join(os.path.dirname(HERE), "include", "nova_attn.h"))
+    deps.append(os.path.join(os.path.dirname(HERE), "include", "nova_lmhead.h"))
     return any(os.path.getmtime(d) > t for d in deps)
 
 

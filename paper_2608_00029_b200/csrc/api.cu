@@ -11,6 +11,7 @@
 #include <mutex>
 
 #include "../../include/nova_attn.h"
+#include "../../include/nova_lmhead.h"
 #include "kernels.h"
 
 namespace nova {
@@ -76,6 +77,7 @@ int device_state(DeviceState** out) {
         if (e == cudaSuccess) e = configure_attn_bwd();
         if (e == cudaSuccess) e = configure_attn_delta();
         if (e == cudaSuccess) e = configure_attn_dq();
+        if (e == cudaSuccess) e = configure_lmhead();
         if (e == cudaSuccess) e = cudaGetSymbolAddress(reinterpret_cast<void**>(&st.dev_status), g_dev_status);
         if (e != cudaSuccess) { st.status = fail_cuda(e); return st.status; }
     }
@@ -197,6 +199,25 @@ int get_tensor_map4(const void* ptr, const AttnShape& s, const TensorStrides& st
     e.valid = true;
     *out = m;
     *order = static_cast<uint32_t>(code);
+    return NOVA_ATTN_OK;
+}
+
+// 2-D map of a row-major bf16 matrix [rows, cols] (cols contiguous): dimensions [cols, rows], box
+// [box_cols, box_rows], 128-byte swizzle; elements outside the matrix read as zeros.
+int encode_matrix_map(const void* ptr, long long rows, long long cols, int box_rows, int box_cols, CUtensorMap* out) {
+    const cuuint64_t dims[2] = {cuuint64_t(cols), cuuint64_t(rows)};
+    const cuuint64_t strides[1] = {cuuint64_t(cols) * sizeof(__nv_bfloat16)};
+    const cuuint32_t box[2] = {cuuint32_t(box_cols), cuuint32_t(box_rows)};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = g_encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? NOVA_ATTN_OK : fail_cuda(static_cast<int>(r));
+}
+
+int check_lmhead_shape(int M, int N, int K) {
+    if (M <= 0 || N <= 0 || K <= 0 || (K & 7) || (N & 7)) return NOVA_ATTN_ERR_SHAPE;
+    if (M > (1 << 28) || N > (1 << 28) || K > (1 << 20)) return NOVA_ATTN_ERR_SHAPE;
     return NOVA_ATTN_OK;
 }
 
@@ -468,6 +489,38 @@ int nova_attn_bwd_strided(const void* Q, const void* K, const void* V, const voi
     return bwd_impl(Q, K, V, dO, LSE, Delta, dQ, dK, dV, B, H, T, D, sq, sk, sv, sdo, sdq, sdk, sdv, scale, causal,
                     workspace, workspace_bytes, stream,
                     NOVA_ATTN_BWD_STEP_ZERO | NOVA_ATTN_BWD_STEP_MAIN | NOVA_ATTN_BWD_STEP_CONVERT);
+}
+
+size_t nova_lmhead_workspace_bytes(int M, int N, int K) {
+    if (check_lmhead_shape(M, N, K) != NOVA_ATTN_OK) return 0;
+    return lmhead_workspace_bytes(M, N);
+}
+
+int nova_lmhead_fwd(const void* X, const void* W, const int* targets, void* logits, float* lse, float* loss, int M,
+                    int N, int K, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!X || !W || !targets || !lse || !loss) return NOVA_ATTN_ERR_NULL;
+    if (int rc = check_lmhead_shape(M, N, K)) return rc;
+    if (!aligned16(X) || !aligned16(W) || !aligned16(logits)) return NOVA_ATTN_ERR_ALIGNMENT;
+    if ((reinterpret_cast<uintptr_t>(targets) & 3u) || (reinterpret_cast<uintptr_t>(lse) & 3u) ||
+        (reinterpret_cast<uintptr_t>(loss) & 3u))
+        return NOVA_ATTN_ERR_ALIGNMENT;
+    if (!workspace || workspace_bytes < lmhead_workspace_bytes(M, N)) return NOVA_ATTN_ERR_WORKSPACE;
+    if (!aligned16(workspace)) return NOVA_ATTN_ERR_ALIGNMENT;
+    DeviceState* st = nullptr;
+    if (int rc = device_state(&st)) return rc;
+    int rows_x = 0, rows_w = 0;
+    const int box_k = lmhead_boxes(&rows_x, &rows_w);
+    CUtensorMap tmX, tmW, tmL;
+    if (int rc = encode_matrix_map(X, M, K, rows_x, box_k, &tmX)) return rc;
+    if (int rc = encode_matrix_map(W, N, K, rows_w, box_k, &tmW)) return rc;
+    if (logits) {
+        if (int rc = encode_matrix_map(logits, M, N, 32, 64, &tmL)) return rc;
+    } else {
+        tmL = tmX;  // never used
+    }
+    const cudaError_t e = launch_lmhead(tmX, tmW, tmL, logits != nullptr, targets, lse, loss, M, N, K, workspace,
+                                        st->num_sms, st->dev_status, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? NOVA_ATTN_OK : fail_cuda(e);
 }
 
 const char* nova_attn_status_string(int status) {

@@ -31,6 +31,29 @@ def test_header_symbols_are_exported(lib):
         assert hasattr(lib, n), f"{n} declared in nova_attn.h but not exported"
 
 
+def test_loss_head_header_symbols_and_validation(lib):
+    """include/nova_lmhead.h: every declared entry point is exported, and bad arguments are rejected on the host."""
+    from paper_2608_00029_b200 import nova_attn as na, nova_lmhead as lm
+    text = re.sub(r"/\*.*?\*/", "", open(os.path.join(ROOT, "include", "nova_lmhead.h")).read(), flags=re.S)
+    names = sorted(set(re.findall(r"\b(nova_lmhead_[a-z_0-9]+)\s*\(", text)))
+    assert names == ["nova_lmhead_fwd", "nova_lmhead_workspace_bytes"]
+    for n in names:
+        assert hasattr(lib, n), f"{n} declared in nova_lmhead.h but not exported"
+    assert lm.nova_lmhead_workspace_bytes(8192, 50304, 768) == 393 * 8192 * 8 + 8192 * 4
+    assert lm.nova_lmhead_workspace_bytes(1, 8, 8) == 256
+    assert lm.nova_lmhead_workspace_bytes(8, 12, 8) == 0 and lm.nova_lmhead_workspace_bytes(8, 16, 12) == 0
+    p = ctypes.c_void_p(0x1000)
+    f = lm._lib().nova_lmhead_fwd
+    assert f(None, p, p, p, p, p, 8, 8, 8, p, 1 << 20, None) == na.ERR_NULL
+    assert f(p, p, p, None, p, None, 8, 8, 8, p, 1 << 20, None) == na.ERR_NULL      # loss is required, logits are not
+    assert f(p, p, p, p, p, p, 0, 8, 8, p, 1 << 20, None) == na.ERR_SHAPE
+    assert f(p, p, p, p, p, p, 8, 12, 8, p, 1 << 20, None) == na.ERR_SHAPE           # N not a multiple of 8
+    assert f(p, p, p, p, p, p, 8, 8, 4, p, 1 << 20, None) == na.ERR_SHAPE
+    assert f(p, ctypes.c_void_p(0x1008), p, p, p, p, 8, 8, 8, p, 1 << 20, None) == na.ERR_ALIGNMENT
+    assert f(p, p, p, p, p, p, 8, 8, 8, None, 0, None) == na.ERR_WORKSPACE
+    assert f(p, p, p, p, p, p, 8, 8, 8, p, 16, None) == na.ERR_WORKSPACE
+
+
 def test_status_strings(lib):
     from paper_2608_00029_b200 import nova_attn as na
     assert na.nova_attn_status_string(0) == "ok"
