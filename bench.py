@@ -338,6 +338,166 @@ def run_grid(args):
     return 0
 
 
+def run_lmhead(args):
+    """The second workload: the fused loss head (projection + softmax cross-entropy statistics + merge) on the
+    paper's shape.  One step = one nova_lmhead_fwd call; value = projection TFLOP/s (2*M*N*K)."""
+    from paper_2608_00029_b200 import nova_attn as na, nova_lmhead as lm
+    na.load()
+    rank, local_rank, world = multi.env_rank_world()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the loss head has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        multi.init_process_group("nccl")
+    peaks, peak_src = load_peaks()
+    cfg = W.LM_HEAD_CONFIGS[args.workload]  # rows are independent: every rank runs the same number of rows
+    stream = torch.cuda.current_stream()
+
+    def make_set(seed):
+        X, Wm, t = (a.to(dev) for a in W.make_lmhead_inputs(cfg, seed=seed))
+        return {"X": X, "W": Wm, "t": t, "logits": torch.empty((cfg.M, cfg.N), dtype=torch.bfloat16, device=dev),
+                "lse": torch.empty(cfg.M, dtype=torch.float32, device=dev),
+                "loss": torch.empty(cfg.M, dtype=torch.float32, device=dev),
+                "ws": torch.empty(lm.nova_lmhead_workspace_bytes(cfg.M, cfg.N, cfg.K), dtype=torch.uint8, device=dev)}
+
+    sets = [make_set(cfg.seed + 1000 * rank + i) for i in range(2)]  # each set (logits alone 0.8 GB) exceeds L2
+    set_bytes = sum(v.numel() * v.element_size() for v in sets[0].values())
+
+    def step(s):
+        lm.nova_lmhead_fwd(s["X"], s["W"], s["t"], s["logits"], s["lse"], s["loss"], s["ws"])
+
+    if args.profile:
+        for i in range(args.warmup + args.steps):
+            step(sets[0])
+        na.nova_attn_poll_device_status()
+        print(json.dumps({"profile_run": cfg.name, "M": cfg.M, "N": cfg.N, "K": cfg.K, "steps": args.warmup + args.steps,
+                          "checksum": float(sets[0]["loss"].sum())}), flush=True)
+        return 0
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    for i in range(max(args.warmup, 3)):
+        step(sets[i % 2])
+    torch.cuda.synchronize()
+    multi.barrier()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    ev0.record(stream)
+    for i in range(args.steps):
+        step(sets[i % 2])
+    ev1.record(stream)
+    torch.cuda.synchronize()
+    t1 = time.perf_counter()
+    multi.barrier()
+    ms = multi.max_over_ranks(ev0.elapsed_time(ev1), dev) / args.steps
+    na.nova_attn_poll_device_status()
+    value = cfg.flops * world / (ms * 1e-3) / 1e12
+
+    # the contraction kernel alone (it is followed at once by the merge: time the pair, then the pair without
+    # the logits, which removes the only large store)
+    def timed(fn, n):
+        for i in range(3):
+            fn(sets[i % 2])
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for i in range(n):
+            fn(sets[i % 2])
+        b.record(stream)
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / n
+
+    n_attr = min(args.steps, 50)
+    ms_nolog = timed(lambda s: lm.nova_lmhead_fwd(s["X"], s["W"], s["t"], None, s["lse"], s["loss"], s["ws"]), n_attr)
+
+    # context only: the same chain as three library calls (projection, log-softmax pass, NLL pick)
+    def library_chain(s):
+        z = torch.matmul(s["X"], s["W"].T, out=s["logits"])
+        return torch.logsumexp(z, dim=1)
+
+    try:
+        ms_lib_gemm = timed(lambda s: torch.matmul(s["X"], s["W"].T, out=s["logits"]), n_attr)
+        ms_lib_chain = timed(library_chain, n_attr)
+    except Exception:
+        ms_lib_gemm = ms_lib_chain = None
+
+    # end to end: the step's hidden states and targets come from pinned host memory, its losses go back
+    hX = [sets[i]["X"].cpu().pin_memory() for i in range(2)]
+    hT = [sets[i]["t"].cpu().pin_memory() for i in range(2)]
+    hOut = [torch.empty((2, cfg.M), dtype=torch.float32).pin_memory() for _ in range(2)]
+
+    def e2e_step(i):
+        s = sets[i % 2]
+        s["X"].copy_(hX[i % 2], non_blocking=True)
+        s["t"].copy_(hT[i % 2], non_blocking=True)
+        step(s)
+        hOut[i % 2][0].copy_(s["lse"], non_blocking=True)
+        hOut[i % 2][1].copy_(s["loss"], non_blocking=True)
+
+    n_e2e = max(3, min(args.steps, 50))
+    for i in range(3):
+        e2e_step(i)
+    torch.cuda.synchronize()
+    multi.barrier()
+    ev0.record(stream)
+    for i in range(n_e2e):
+        e2e_step(i)
+    ev1.record(stream)
+    torch.cuda.synchronize()
+    multi.barrier()
+    e2e_ms = multi.max_over_ranks(ev0.elapsed_time(ev1), dev) / n_e2e
+    sampler.stop()
+    sampler.join(timeout=2)
+
+    cpu_baseline = None
+    if rank == 0 and world == 1:
+        import oracle
+        oracle.build()
+        X, Wm, t = W.make_lmhead_inputs(cfg)
+        Wd = W.widen(Wm)
+        rows, spent = 0, 0.0
+        chunk = 48
+        while spent < 10.0 and rows < cfg.M:
+            tt = time.perf_counter()
+            oracle.lmhead_fwd(W.widen(X[rows:rows + chunk]), Wd, t[rows:rows + chunk].numpy())
+            spent += time.perf_counter() - tt
+            rows += chunk
+        cpu_baseline = {"value": 2.0 * rows * cfg.N * cfg.K / spent / 1e12, "unit": UNIT, "cores": oracle.num_threads(),
+                        "kind": "oracle", "sample": f"{rows} of {cfg.M} rows of {cfg.name}, {spent:.2f} s"}
+
+    if rank == 0:
+        peak = peaks["bf16_tflops"]
+        ach = cfg.flops / (ms * 1e-3) / 1e12
+        line = {
+            "metric": "lm_head_fused_tflops", "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": cfg.name, "M": cfg.M, "N": cfg.N, "K": cfg.K, "logits": "bf16, stored",
+                       "parallelism": f"dp{world} (rows split, no collective)",
+                       "l2": f"alternating 2 buffer sets of {set_bytes / 1e6:.0f} MB (> 126 MB L2)",
+                       "launch": "eager (2 kernels per step)",
+                       "context": "the paper's fused loss head takes 7.91 ms on an RTX 6000 Ada (TF32, fp32 logits)"},
+            "e2e": {"value": cfg.flops * world / (e2e_ms * 1e-3) / 1e12, "unit": UNIT,
+                    "h2d_bytes_per_step": int(hX[0].numel() * 2 + hT[0].numel() * 4), "d2h_bytes_per_step": int(cfg.M * 8),
+                    "ms_per_step": e2e_ms, "steps": n_e2e},
+            "gpu_launches": 2 * args.steps,
+            "clocks": sampler.summary(t0, t1),
+            "roofline": {"bound": "tensor", "kernel": "lmhead_kernel (+ lmhead_merge_kernel)", "achieved": ach, "peak": peak,
+                         "unit": UNIT, "frac": ach / peak, "traffic": None, "peak_source": f"{peak_src} bf16_tflops (burst)",
+                         "ms_per_launch": ms, "ms_without_logits": ms_nolog,
+                         "library_context": {"what": "torch.matmul alone / torch.matmul + logsumexp over the stored logits",
+                                             "ms_gemm": ms_lib_gemm, "ms_gemm_plus_reduction": ms_lib_chain}},
+            "cpu_baseline": cpu_baseline,
+        }
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        multi.barrier()
+        torch.distributed.destroy_process_group()
+    return 0
+
+
 def run_ours(args):
     from paper_2608_00029_b200 import nova_attn as na
     na.load()  # fails loudly if the CUDA library has not been built
@@ -602,7 +762,7 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--launch", choices=["graph", "eager"], default="graph",
                     help="timed steps replayed from a CUDA graph per buffer set (default) or issued call by call")
-    ap.add_argument("--workload", choices=W.CONFIG_ORDER, default=WORKLOAD,
+    ap.add_argument("--workload", choices=W.CONFIG_ORDER + sorted(W.LM_HEAD_CONFIGS), default=WORKLOAD,
                     help="the configuration to run (the headline number is quoted on the default)")
     ap.add_argument("--profile", action="store_true",
                     help="only run warmup + steps steps on one buffer set and exit: a short command for a profiler")
@@ -614,6 +774,12 @@ def main():
         if args.steps == 500:
             args.steps = 30
         return run_grid(args)
+    if args.workload in W.LM_HEAD_CONFIGS:
+        if args.impl == "reference":
+            raise SystemExit("--impl reference times the attention oracle: use an attention workload")
+        if args.steps == 500:
+            args.steps = 100
+        return run_lmhead(args)
     if args.impl == "reference":
         return run_reference(args)
     return run_ours(args)
