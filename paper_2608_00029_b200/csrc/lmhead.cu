@@ -287,33 +287,49 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ C
 
 // Merge of the partial statistics of each row (paper Section 4.1: "a running maximum and a running sum do not
 // combine via the same operation that accumulates them"): the pair with the smaller maximum has its sum
-// multiplied by exp(smaller - larger) before the sums are added.  One thread per row; the partials of
-// consecutive rows are adjacent, so a warp reads 256 contiguous bytes per step.
-__global__ void __launch_bounds__(64)
+// multiplied by exp(smaller - larger) before the sums are added.  A block takes 32 rows; its 8 warps each walk
+// every eighth partial of those rows (the partials of consecutive rows are adjacent, so a warp reads 256
+// contiguous bytes per step, many steps in flight), and the 8 intermediate pairs of a row are merged by the
+// same rule through shared memory.
+constexpr int kMergeRows = 32, kMergeSlices = 8;
+
+__device__ __forceinline__ void merge_pair(float& m, float& l, float m2, float l2) {
+    if (l2 > 0.f) {
+        if (m2 > m) {
+            l = l * __expf(m - m2) + l2;  // exp(-inf) = 0 while nothing has been merged yet
+            m = m2;
+        } else {
+            l += l2 * __expf(m2 - m);
+        }
+    }
+}
+
+__global__ void __launch_bounds__(kMergeRows * kMergeSlices)
 lmhead_merge_kernel(const float2* __restrict__ partials, const float* __restrict__ tgt_logit,
                     const int* __restrict__ targets, float* __restrict__ lse, float* __restrict__ loss, int M, int N,
                     int n_part) {
+    __shared__ float2 inter[kMergeSlices][kMergeRows];
     griddep_launch_dependents();
     griddep_wait();
-    const int row = blockIdx.x * blockDim.x + threadIdx.x;
-    if (row >= M) return;
+    const int rl = threadIdx.x % kMergeRows, slice = threadIdx.x / kMergeRows;
+    const int row = blockIdx.x * kMergeRows + rl;
     float m = -INFINITY, l = 0.f;
+    if (row < M) {
 #pragma unroll 8
-    for (int p = 0; p < n_part; ++p) {
-        const float2 q = partials[static_cast<size_t>(p) * M + row];
-        if (q.y > 0.f) {
-            if (q.x > m) {
-                l = l * __expf(m - q.x) + q.y;  // exp(-inf) = 0 the first time
-                m = q.x;
-            } else {
-                l += q.y * __expf(q.x - m);
-            }
+        for (int p = slice; p < n_part; p += kMergeSlices) {
+            const float2 q = partials[static_cast<size_t>(p) * M + row];
+            merge_pair(m, l, q.x, q.y);
         }
     }
-    const float v = m + logf(l);
-    const int t = targets[row];
-    lse[row] = v;
-    loss[row] = (t >= 0 && t < N) ? v - tgt_logit[row] : 0.f;
+    inter[slice][rl] = make_float2(m, l);
+    __syncthreads();
+    if (slice == 0 && row < M) {
+        for (int s = 1; s < kMergeSlices; ++s) merge_pair(m, l, inter[s][rl].x, inter[s][rl].y);
+        const float v = m + logf(l);
+        const int t = targets[row];
+        lse[row] = v;
+        loss[row] = (t >= 0 && t < N) ? v - tgt_logit[row] : 0.f;
+    }
 }
 
 }  // namespace
@@ -339,7 +355,8 @@ cudaError_t launch_lmhead(const CUtensorMap& tmX, const CUtensorMap& tmW, const 
     cudaError_t e = launch_overlapped(lmhead_kernel, grid, dim3(kThreads), kSmemBytes, stream, tmX, tmW, tmL, targets,
                                       store_logits ? 1 : 0, partials, tgt_logit, M, N, K, dev_status);
     if (e != cudaSuccess) return e;
-    return launch_overlapped(lmhead_merge_kernel, dim3((M + 63) / 64), dim3(64), 0, stream,
+    return launch_overlapped(lmhead_merge_kernel, dim3((M + kMergeRows - 1) / kMergeRows),
+                             dim3(kMergeRows * kMergeSlices), 0, stream,
                              static_cast<const float2*>(partials), static_cast<const float*>(tgt_logit), targets, lse, loss,
                              M, N, n_part);
 }
