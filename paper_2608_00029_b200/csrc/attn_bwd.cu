@@ -45,9 +45,7 @@
 namespace nova {
 namespace {
 
-constexpr int kBwdThreads = 512;
 constexpr int kBwdTmemCols = 512;
-constexpr int kComputeWarps = 8;
 
 template <int D>
 struct BwdCfg {
@@ -86,7 +84,12 @@ struct BwdCfg {
     static constexpr bool kSeparateP = (D == 64);   // P^T in its own columns instead of over S^T
     static constexpr int kColP = kSeparateP ? 448 : 0;
     static constexpr int kPHalfStride = kSeparateP ? 32 : 64;  // column distance between the two query halves of P^T
-    static constexpr int kQPT = 64;            // queries per compute thread (128 / kQPT warpgroups of compute warps)
+    // Queries per compute thread: 128 / kQPT warpgroups of compute warps.  Two warpgroups of 64 queries each:
+    // four of 32 (four compute warps per scheduler, 768 threads, 80 registers) were measured 26 % slower at
+    // D=64 (78.3 against 62.1 us on B=8, H=12, T=1024).
+    static constexpr int kQPT = 64;
+    static constexpr int kComputeWarps = 4 * (128 / kQPT);
+    static constexpr int kThreads = 32 * (4 + kComputeWarps + 4);  // producer, UMMA, 2 row loaders, compute, 4 dQ
 };
 
 struct BwdBars {
@@ -312,7 +315,9 @@ __device__ __forceinline__ void bwd_mma(uint8_t* smem, BwdBars* bars, uint32_t t
                 const uint32_t b = q_m0 + (g % Cfg::kQStages) * kQStageStep;
 #pragma unroll
                 for (int k = 0; k < kBlockQ / 16; ++k)
-                    umma_ts(t_dk, t_dp + (k / 4) * 64 + (k % 4) * 8, umma_desc_join(b + k * 128, hi), kIdescKV,
+                    // bf16 dS^T of 16 queries: 8 packed columns at the start of the fp32 columns of their thread
+                    umma_ts(t_dk, t_dp + (k / (Cfg::kQPT / 16)) * Cfg::kQPT + (k % (Cfg::kQPT / 16)) * 8,
+                            umma_desc_join(b + k * 128, hi), kIdescKV,
                             (it > 0 || k > 0) ? 1u : 0u);
                 tc_commit(&bars->q_empty[g % Cfg::kQStages]);
             }
@@ -670,23 +675,25 @@ __device__ __forceinline__ void bwd_dq_tma(uint8_t* smem, BwdBars* bars, uint32_
             ok = mbar_wait(&bars->dq_full, g & 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
-            uint32_t a[64];
-            tmem_ld_x32(t_dq, a);
-            tmem_ld_x32(t_dq + 32, a + 32);
-            tmem_wait_ld();
+            // The staging buffer first (its previous contents were handed to the copy engine a whole tile ago),
+            // then the tile leaves TMEM 32 columns = one box at a time, which keeps the register count down.
+            ok = stage_reusable();
+            if (!ok) break;
+#pragma unroll
+            for (int hb = 0; hb < 2; ++hb) {
+                uint32_t a[32];
+                tmem_ld_x32(t_dq + 32 * hb, a);
+                tmem_wait_ld();
+                uint8_t* rowp = hb ? row1 : row0;
+                // fp32 [128 rows x 32 columns] per box: eight 16-byte chunks per row, 128-byte swizzle
+#pragma unroll
+                for (int ch = 0; ch < 8; ++ch)
+                    *reinterpret_cast<uint4*>(rowp + ((ch ^ sw) << 4)) =
+                        make_uint4(a[ch * 4], a[ch * 4 + 1], a[ch * 4 + 2], a[ch * 4 + 3]);
+            }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&bars->dq_free);
-            ok = stage_reusable();
-            if (!ok) break;
-            // fp32 [128 rows x 32 columns] per box: eight 16-byte chunks per row, 128-byte swizzle
-#pragma unroll
-            for (int ch = 0; ch < 8; ++ch) {
-                *reinterpret_cast<uint4*>(row0 + ((ch ^ sw) << 4)) =
-                    make_uint4(a[ch * 4], a[ch * 4 + 1], a[ch * 4 + 2], a[ch * 4 + 3]);
-                *reinterpret_cast<uint4*>(row1 + ((ch ^ sw) << 4)) =
-                    make_uint4(a[32 + ch * 4], a[32 + ch * 4 + 1], a[32 + ch * 4 + 2], a[32 + ch * 4 + 3]);
-            }
             ok = flush(0, (i0 + it) * kBlockQ, bh);
             if (!ok) break;
         }
@@ -695,37 +702,33 @@ __device__ __forceinline__ void bwd_dq_tma(uint8_t* smem, BwdBars* bars, uint32_
         ok = mbar_wait(&bars->dkv_full, w & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
-        uint32_t pv[32], pk[32];
+        ok = stage_reusable();
+        if (!ok) break;
 #pragma unroll
         for (int cb = 0; cb < 64; cb += 32) {  // 32 accumulator columns at a time keeps the register count down
             uint32_t a[32];
             tmem_ld_x32(t_dv + cb, a);
             tmem_wait_ld();
 #pragma unroll
-            for (int x = 0; x < 16; ++x)
-                pv[cb / 2 + x] = pack_bf16x2(__uint_as_float(a[2 * x]), __uint_as_float(a[2 * x + 1]));
-        }
-#pragma unroll
-        for (int cb = 0; cb < 64; cb += 32) {
-            uint32_t a[32];
+            for (int ch = 0; ch < 4; ++ch)  // 8 bf16 = 16 bytes per chunk
+                *reinterpret_cast<uint4*>(row0 + (((cb / 8 + ch) ^ sw) << 4)) =
+                    make_uint4(pack_bf16x2(__uint_as_float(a[8 * ch + 0]), __uint_as_float(a[8 * ch + 1])),
+                               pack_bf16x2(__uint_as_float(a[8 * ch + 2]), __uint_as_float(a[8 * ch + 3])),
+                               pack_bf16x2(__uint_as_float(a[8 * ch + 4]), __uint_as_float(a[8 * ch + 5])),
+                               pack_bf16x2(__uint_as_float(a[8 * ch + 6]), __uint_as_float(a[8 * ch + 7])));
             tmem_ld_x32(t_dk + cb, a);
             tmem_wait_ld();
 #pragma unroll
-            for (int x = 0; x < 16; ++x)
-                pk[cb / 2 + x] = pack_bf16x2(__uint_as_float(a[2 * x]) * scale, __uint_as_float(a[2 * x + 1]) * scale);
+            for (int ch = 0; ch < 4; ++ch)
+                *reinterpret_cast<uint4*>(row1 + (((cb / 8 + ch) ^ sw) << 4)) = make_uint4(
+                    pack_bf16x2(__uint_as_float(a[8 * ch + 0]) * scale, __uint_as_float(a[8 * ch + 1]) * scale),
+                    pack_bf16x2(__uint_as_float(a[8 * ch + 2]) * scale, __uint_as_float(a[8 * ch + 3]) * scale),
+                    pack_bf16x2(__uint_as_float(a[8 * ch + 4]) * scale, __uint_as_float(a[8 * ch + 5]) * scale),
+                    pack_bf16x2(__uint_as_float(a[8 * ch + 6]) * scale, __uint_as_float(a[8 * ch + 7]) * scale));
         }
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(&bars->dkv_free);
-        ok = stage_reusable();
-        if (!ok) break;
-#pragma unroll
-        for (int ch = 0; ch < 8; ++ch) {
-            *reinterpret_cast<uint4*>(row0 + ((ch ^ sw) << 4)) =
-                make_uint4(pv[ch * 4], pv[ch * 4 + 1], pv[ch * 4 + 2], pv[ch * 4 + 3]);
-            *reinterpret_cast<uint4*>(row1 + ((ch ^ sw) << 4)) =
-                make_uint4(pk[ch * 4], pk[ch * 4 + 1], pk[ch * 4 + 2], pk[ch * 4 + 3]);
-        }
         ok = flush(1, kt * kBlockK, bh);
         ++w;
     }
@@ -814,7 +817,7 @@ __device__ __forceinline__ void bwd_dq_tma_wide(uint8_t* smem, BwdBars* bars, ui
 }
 
 template <int D, bool kCausal, bool kStrided>
-__global__ void __launch_bounds__(kBwdThreads, 1)
+__global__ void __launch_bounds__(BwdCfg<D>::kThreads, 1)
 attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmdO,
                 const __grid_constant__ CUtensorMap tmAcc, const __grid_constant__ CUtensorMap tmdK,
@@ -847,18 +850,18 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             mbar_init(&bars->do_full[s], 1);
             mbar_init(&bars->do_empty[s], 1);
             mbar_init(&bars->row_full[s], 2);
-            mbar_init(&bars->row_empty[s], kComputeWarps);
+            mbar_init(&bars->row_empty[s], Cfg::kComputeWarps);
         }
         mbar_init(&bars->s_full, 1);
         mbar_init(&bars->dp_full, 1);
-        mbar_init(&bars->p_ready, kComputeWarps);
-        mbar_init(&bars->ds_ready, kComputeWarps);
+        mbar_init(&bars->p_ready, Cfg::kComputeWarps);
+        mbar_init(&bars->ds_ready, Cfg::kComputeWarps);
         mbar_init(&bars->dq_full, 1);
         mbar_init(&bars->dq_free, 4);
         mbar_init(&bars->stage_full, 4);
         mbar_init(&bars->stage_free, 1);
         mbar_init(&bars->dkv_full, 1);
-        mbar_init(&bars->dkv_free, Cfg::kBulkdQ ? 4 : kComputeWarps);
+        mbar_init(&bars->dkv_free, Cfg::kBulkdQ ? 4 : Cfg::kComputeWarps);
         mbar_init(&bars->drain, 1);
         bars->abort_flag = 0;
         fence_mbar_init();
@@ -900,13 +903,13 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         bwd_mma<D>(smem, bars, tmem_base, wl);
     } else if (warp < 4) {
         bwd_rows(bars, reinterpret_cast<float*>(smem + Cfg::kOffRow), LSE, Delta, T, wl, (warp - 2) * 32 + lane);
-    } else if (warp < 12) {
+    } else if (warp < 4 + Cfg::kComputeWarps) {
         bwd_compute<D, kCausal>(smem, bars, tmem_base, dK, dV, sdk, sdv, T, scale, wl, warp - 4, lane);
     } else {
         if constexpr (Cfg::kBulkdQ)
-            bwd_dq_tma<kStrided>(smem, bars, tmem_base, &tmAcc, &tmdK, &tmdV, scale, wl, warp - 12, lane);
+            bwd_dq_tma<kStrided>(smem, bars, tmem_base, &tmAcc, &tmdK, &tmdV, scale, wl, warp - 4 - Cfg::kComputeWarps, lane);
         else
-            bwd_dq_tma_wide(smem, bars, tmem_base, &tmAcc, wl, warp - 12, lane);
+            bwd_dq_tma_wide(smem, bars, tmem_base, &tmAcc, wl, warp - 4 - Cfg::kComputeWarps, lane);
     }
 
     tc_fence_before();
@@ -926,10 +929,10 @@ cudaError_t launch_one(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUt
     const long long n_items = static_cast<long long>(n_tiles) * BH;
     const dim3 grid(static_cast<unsigned>(n_items < num_sms ? n_items : num_sms));  // one persistent CTA per SM
     if (strided)
-        return launch_overlapped(attn_bwd_kernel<D, kCausal, true>, grid, dim3(kBwdThreads), BwdCfg<D>::kSmemBytes,
+        return launch_overlapped(attn_bwd_kernel<D, kCausal, true>, grid, dim3(BwdCfg<D>::kThreads), BwdCfg<D>::kSmemBytes,
                                  stream, tmQ, tmK, tmV, tmdO, tmAcc, tmdK, tmdV, LSE, Delta, dK, dV, sdk, sdv, s.T, BH, s.H,
                                  orders, no_dq ? 1 : 0, n_tiles, s.scale, dev_status);
-    return launch_overlapped(attn_bwd_kernel<D, kCausal, false>, grid, dim3(kBwdThreads), BwdCfg<D>::kSmemBytes, stream,
+    return launch_overlapped(attn_bwd_kernel<D, kCausal, false>, grid, dim3(BwdCfg<D>::kThreads), BwdCfg<D>::kSmemBytes, stream,
                              tmQ, tmK, tmV, tmdO, tmAcc, tmdK, tmdV, LSE, Delta, dK, dV, sdk, sdv, s.T, BH, s.H, orders,
                              no_dq ? 1 : 0, n_tiles, s.scale, dev_status);
 }
