@@ -587,45 +587,80 @@ def run_ours(args):
     ms_per_step = ms_total / args.steps
     value = flops_step * world / (ms_per_step * 1e-3) / 1e12
 
-    # ---- per-kernel attribution (separate pass, same rotation): events around each launch
+    # ---- per-kernel attribution.  Two passes over the same rotation of buffer sets:
+    # (1) each kernel's launches recorded back to back into a CUDA graph and replayed, as they run inside the
+    #     timed steps (no host in between): `kernel_ms`, the figure the roofline uses;
+    # (2) the calls issued one by one with an event on either side: `kernel_ms_eager`.  The host needs longer to
+    #     issue a launch and two event records than these kernels run, so this figure contains idle time.
     names = ["fwd", "bwd_preprocess", "bwd_zero", "bwd_main", "bwd_convert"]
+
+    def one_kernel(name, s):
+        if name == "fwd":
+            na.nova_attn_fwd(s.q, s.k, s.v, s.o, s.lse, cfg.scale, cfg.causal)
+        elif name == "bwd_preprocess":
+            na.nova_attn_bwd_preprocess(s.o, s.do, s.delta)
+        elif name == "bwd":  # the whole backward as the three calls make it: preprocess + clear + main + convert
+            na.nova_attn_bwd_preprocess(s.o, s.do, s.delta)
+            na.nova_attn_bwd(s.q, s.k, s.v, s.o, s.do, s.lse, s.delta, s.dq, s.dk, s.dv, cfg.scale, cfg.causal, s.ws)
+        else:
+            bit = {"bwd_zero": na.BWD_STEP_ZERO, "bwd_main": na.BWD_STEP_MAIN, "bwd_convert": na.BWD_STEP_CONVERT}[name]
+            na.nova_attn_bwd(s.q, s.k, s.v, s.o, s.do, s.lse, s.delta, s.dq, s.dk, s.dv, cfg.scale, cfg.causal, s.ws,
+                             steps=bit)
+
+    def graph_ms(name, rounds=8, reps=5):
+        """Mean duration of `name`, launched rounds * n_sets times back to back from a CUDA graph."""
+        side = torch.cuda.Stream(device=dev)
+        with torch.cuda.stream(side):
+            for s in sets:
+                one_kernel(name, s)
+        side.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side, capture_error_mode="thread_local"):
+            for _ in range(rounds):
+                for s in sets:
+                    one_kernel(name, s)
+        g.replay()
+        torch.cuda.synchronize()
+        times = []
+        for _ in range(reps):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            g.replay()
+            b.record(stream)
+            torch.cuda.synchronize()
+            times.append(a.elapsed_time(b) / (rounds * n_sets))
+        return sorted(times)[len(times) // 2]
+
+    attribution = "CUDA graph of back-to-back launches per kernel"
+    try:
+        kernel_ms = {n: graph_ms(n) for n in names}
+        fwd_seq_ms, bwd_seq_ms = kernel_ms["fwd"], graph_ms("bwd")
+    except Exception as e:  # capture unavailable: fall back to the eager figures and say so
+        print(f"bench.py: per-kernel graph capture failed ({e!r}); using eager launches", file=sys.stderr)
+        torch.cuda.synchronize()
+        kernel_ms = None
+        attribution = "eager launches between events (contains host gaps)"
+
     k_steps = min(args.steps, 200)
     evs = [[torch.cuda.Event(enable_timing=True) for _ in range(len(names) + 1)] for _ in range(k_steps)]
     for i in range(k_steps):
         s = sets[i % n_sets]
         e = evs[i]
         e[0].record(stream)
-        na.nova_attn_fwd(s.q, s.k, s.v, s.o, s.lse, cfg.scale, cfg.causal)
-        e[1].record(stream)
-        na.nova_attn_bwd_preprocess(s.o, s.do, s.delta)
-        e[2].record(stream)
-        for n, bit in enumerate((na.BWD_STEP_ZERO, na.BWD_STEP_MAIN, na.BWD_STEP_CONVERT)):
-            na.nova_attn_bwd(s.q, s.k, s.v, s.o, s.do, s.lse, s.delta, s.dq, s.dk, s.dv, cfg.scale, cfg.causal, s.ws,
-                             steps=bit)
-            e[3 + n].record(stream)
+        for j, n in enumerate(names):
+            one_kernel(n, s)
+            e[j + 1].record(stream)
     torch.cuda.synchronize()
-    kernel_ms = {n: sum(e[i].elapsed_time(e[i + 1]) for e in evs) / k_steps for i, n in enumerate(names)}
-
-    # ---- forward, and the whole backward as one sequence (preprocess + clear + main + convert), each
-    # bracketed by events: what the 50 % / 35 % targets are stated on
-    evq = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(k_steps)]
-    for i in range(k_steps):
-        s = sets[i % n_sets]
-        e = evq[i]
-        e[0].record(stream)
-        na.nova_attn_fwd(s.q, s.k, s.v, s.o, s.lse, cfg.scale, cfg.causal)
-        e[1].record(stream)
-        na.nova_attn_bwd_preprocess(s.o, s.do, s.delta)
-        na.nova_attn_bwd(s.q, s.k, s.v, s.o, s.do, s.lse, s.delta, s.dq, s.dk, s.dv, cfg.scale, cfg.causal, s.ws)
-        e[2].record(stream)
-    torch.cuda.synchronize()
-    fwd_seq_ms = sum(e[0].elapsed_time(e[1]) for e in evq) / k_steps
-    bwd_seq_ms = sum(e[1].elapsed_time(e[2]) for e in evq) / k_steps
+    kernel_ms_eager = {n: sum(e[i].elapsed_time(e[i + 1]) for e in evs) / k_steps for i, n in enumerate(names)}
+    if kernel_ms is None:
+        kernel_ms = kernel_ms_eager
+        fwd_seq_ms = kernel_ms["fwd"]
+        bwd_seq_ms = sum(kernel_ms[n] for n in names[1:])
 
     bwd_ms = kernel_ms["bwd_main"]
     achieved = cfg.bwd_flops / (bwd_ms * 1e-3) / 1e12
-    # every launch of these passes is timed on its own, between events, at full clocks: the burst figure
-    # is the peak that applies; the sustained one is given beside it
+    # these passes are a few milliseconds of work at full clocks: the burst figure is the peak that applies;
+    # the sustained one is given beside it
     peak = peaks["bf16_tflops"]
     fwd_tflops = cfg.fwd_flops / (fwd_seq_ms * 1e-3) / 1e12
     bwd_tflops = cfg.bwd_flops / (bwd_seq_ms * 1e-3) / 1e12
@@ -635,7 +670,7 @@ def run_ours(args):
         "peak_source": f"{peak_src} bf16_tflops (burst)",
         "peak_sustained": peaks["bf16_tflops_sustained"],
         "frac_of_sustained_peak": achieved / peaks["bf16_tflops_sustained"], "ms_per_launch": bwd_ms,
-        "kernel_ms": kernel_ms,
+        "kernel_ms": kernel_ms, "kernel_ms_eager": kernel_ms_eager, "attribution": attribution,
         "targets": {
             "fwd": {"what": "nova_attn_fwd", "ms": fwd_seq_ms, "tflops": fwd_tflops, "frac": fwd_tflops / peak,
                     "target": 0.50},

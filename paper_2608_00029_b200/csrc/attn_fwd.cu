@@ -2,9 +2,12 @@
 // base-2 online softmax, value contraction, causal loop clamp, 1/sum epilogue, LSE saved).
 //
 // A work item is a block of 256 query rows of one (batch, head): two 128-row query tiles, A and B,
-// that share every K/V tile they both need.  The kernel is persistent: one CTA per SM walks a fixed
-// list of items, heaviest first (the last query block of a causal problem sees every key tile),
-// dealt out in zig-zag order.  Roles (384 threads):
+// that share every K/V tile they both need.  The kernel is persistent and its work is handed out
+// dynamically: the grid has one CTA per item, heaviest first (the last query block of a causal problem
+// sees every key tile); one CTA per SM starts, and each, while it works on an item, asks the hardware to
+// cancel the launch of the next CTA that has not started and takes over its item (cluster launch control),
+// so no SM idles while items are left.  The producer warp makes the request and passes the item number to
+// the other roles through a two-entry ring in shared memory.  Roles (384 threads):
 //   warp 0       TMA producer: Q tiles per item, K and V tiles through mbarrier-guarded rings
 //   warp 1       UMMA issuer:  S_t = Q_t K^T  (operands in shared memory, accumulator in TMEM)
 //                              O_t += P_t V   (P read from TMEM as bf16, V from shared memory)
@@ -59,30 +62,41 @@ struct FwdBars {
     uint64_t k_full[2], k_empty[2], v_full[2], v_empty[2];
     uint64_t s_full[2], s_free[2], p_ready[2], pv_done[2], o_free[2], o_staged[2];  // per query tile
     uint64_t drain;
+    uint64_t work_full[2], work_empty[2];  // ring of item numbers: producer -> UMMA issuer and softmax warps
+    uint64_t clc_bar;                      // the answer to a cancellation request has arrived
+    uint4 clc_response;
+    int work_item[2];
     uint32_t tmem_base;
     int abort_flag;
 };
+constexpr int kWorkConsumers = 1 + 8;  // UMMA issuer warp + 8 softmax warps
 
-// This CTA's list of work items: 256-row query blocks, heaviest first, dealt in zig-zag passes.
+// Work items: 256-row query blocks, numbered heaviest first.
 struct FwdWork {
-    int n_items, n_ctas, cta, BH, n_blocks, n_kv_all, T, H;
+    int n_items, BH, n_blocks, n_kv_all, T, H;
     uint32_t orders;  // coordinate orders of the Q, K, V, O tensor maps, four bits each
     bool causal;
-    __device__ __forceinline__ int passes() const { return (n_items + n_ctas - 1) / n_ctas; }
-    // Item of pass p: block index, head, and the number of key tiles each query tile visits
+    // Item `idx`: block index, head, and the number of key tiles each query tile visits
     // (0 if the tile lies entirely past the end of the sequence).
-    __device__ __forceinline__ bool get(int p, int* blk, int* bh, int* n_a, int* n_b) const {
-        const int idx = p * n_ctas + ((p & 1) ? (n_ctas - 1 - cta) : cta);
-        if (idx >= n_items) return false;
+    __device__ __forceinline__ void get(int idx, int* blk, int* bh, int* n_a, int* n_b) const {
         *blk = n_blocks - 1 - idx / BH;
         *bh = idx % BH;
         const int qt_a = 2 * (*blk), qt_b = qt_a + 1;
         // causal clamp of the key loop: tile qt visits key tiles 0..qt
         *n_a = causal ? min(qt_a + 1, n_kv_all) : n_kv_all;
         *n_b = (qt_b * kBlockQ < T) ? (causal ? min(qt_b + 1, n_kv_all) : n_kv_all) : 0;
-        return true;
     }
 };
+
+// Consumer side of the item ring: the number of the w-th item of this CTA, -1 when there are no more, -2 if
+// the wait was given up.  Every lane of the calling warp gets the same answer.
+__device__ __forceinline__ int next_item(FwdBars* bars, int w, int lane, long long limit) {
+    if (!mbar_wait(&bars->work_full[w & 1], (w >> 1) & 1, &bars->abort_flag, limit)) return -2;
+    const int item = *reinterpret_cast<volatile int*>(&bars->work_item[w & 1]);
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&bars->work_empty[w & 1]);
+    return item;
+}
 
 template <int D, bool kStrided>
 __device__ __forceinline__ void fwd_producer(const CUtensorMap* tmQ, const CUtensorMap* tmK,
@@ -93,9 +107,17 @@ __device__ __forceinline__ void fwd_producer(const CUtensorMap* tmQ, const CUten
     int armed_q[2] = {-1, -1}, armed_k[2] = {-1, -1}, armed_v[2] = {-1, -1};
     bool ok = true;
     int w = 0, g = 0;  // items and key tiles loaded so far
-    for (int p = 0; p < wk.passes() && ok; ++p) {
+    int item = blockIdx.x;
+    bool clc_pending = false;
+    for (;;) {
+        // hand the item (or the end mark) to the other roles
+        ok = mbar_wait(&bars->work_empty[w & 1], ((w >> 1) & 1) ^ 1, abort_flag, limit);
+        if (!ok) break;
+        bars->work_item[w & 1] = item;
+        mbar_arrive(&bars->work_full[w & 1]);
+        if (item < 0) break;
         int blk, bh, n_a, n_b;
-        if (!wk.get(p, &blk, &bh, &n_a, &n_b)) continue;
+        wk.get(item, &blk, &bh, &n_a, &n_b);
         const int head = kStrided ? bh % wk.H : 0, batch = kStrided ? bh / wk.H : 0;
         const int qs = w % Cfg::kQStages;
         const uint32_t qph = (w / Cfg::kQStages) & 1;
@@ -135,11 +157,23 @@ __device__ __forceinline__ void fwd_producer(const CUtensorMap* tmQ, const CUten
                 tma_load_tile<kStrided>(smem + Cfg::kOffV + st * Cfg::kTileBytes + h * kHalfTileBytes, tmV, &bars->v_full[st],
                               (wk.orders >> 8) & 15, h * kBoxCols, j * kBlockK, head, batch, bh);
         }
+        if (!ok) break;
+        // All loads of this item are on their way (the other roles are about two key tiles behind): only now
+        // ask for the next item, so that an item is claimed as late as possible and the CTAs that finish early
+        // find the remaining ones.
+        mbar_expect_tx(&bars->clc_bar, 16);
+        clc_try_cancel(&bars->clc_response, &bars->clc_bar);
+        clc_pending = true;
+        ok = mbar_wait(&bars->clc_bar, w & 1, abort_flag, limit);
+        if (!ok) break;
+        clc_pending = false;
+        item = clc_cancelled_cta(&bars->clc_response);
         ++w;
     }
     if (!ok) {
         // Giving up: let the copies already in flight land before the CTA's shared memory goes away.
         int none = 0;
+        if (clc_pending) (void)mbar_wait(&bars->clc_bar, w & 1, &none);  // the answer must land before the CTA ends
         for (int s = 0; s < 2; ++s) {
             if (armed_q[s] >= 0) (void)mbar_wait(&bars->q_full[s], armed_q[s], &none);
             if (armed_k[s] >= 0) (void)mbar_wait(&bars->k_full[s], armed_k[s], &none);
@@ -166,6 +200,7 @@ __device__ __forceinline__ void fwd_mma(uint8_t* smem, FwdBars* bars, uint32_t t
     uint32_t q_k[2] = {0, 0};  // per item: the two query tiles
     // The whole warp runs this role in uniform control flow; one elected lane issues.
     const bool el = elect_one();
+    const int lane = threadIdx.x & 31;
     bool ok = true;
     int w = 0, g = 0;
     int c[2] = {0, 0};   // key tiles processed so far per query tile (phases of its barriers)
@@ -174,7 +209,7 @@ __device__ __forceinline__ void fwd_mma(uint8_t* smem, FwdBars* bars, uint32_t t
 
     // S_t = Q_t K^T for the key tile in stage gk & 1: both operands K-major, 16 head-dim elements
     // (32 bytes) per instruction.
-    auto issue_qk = [&](int t, int gk) {
+    auto issue_qk = [&](int t, int gk, uint32_t q_desc) {
         const uint32_t t_s = tmem_base + Cfg::kColS + 128 * t;
         const uint32_t b = k_k[gk & 1];
         if (Cfg::kSepP && cq[t] > 0) {  // the softmax warps must have read the previous S_t
@@ -187,7 +222,7 @@ __device__ __forceinline__ void fwd_mma(uint8_t* smem, FwdBars* bars, uint32_t t
 #pragma unroll
             for (int k = 0; k < D / 16; ++k) {
                 const uint32_t off = ((k / 4) * kHalfTileBytes + (k % 4) * 32) >> 4;
-                umma_ss(t_s, umma_desc_join(q_k[t] + off, hi), umma_desc_join(b + off, hi), kIdescQK,
+                umma_ss(t_s, umma_desc_join(q_desc + off, hi), umma_desc_join(b + off, hi), kIdescQK,
                         k > 0 ? 1u : 0u);
             }
             tc_commit(&bars->s_full[t]);
@@ -195,26 +230,38 @@ __device__ __forceinline__ void fwd_mma(uint8_t* smem, FwdBars* bars, uint32_t t
         __syncwarp();
     };
 
-    for (int p = 0; p < wk.passes() && ok; ++p) {
+    constexpr int kNotPeeked = -3;
+    int peeked = kNotPeeked;  // the next item's number, if it was looked at from inside the current item
+    bool first_queued = false;  // ... and its first Q K^T products were queued from there
+    for (;;) {
+        const int item = (peeked != kNotPeeked) ? peeked : next_item(bars, w, lane, limit);
+        peeked = kNotPeeked;
+        if (item < 0) {
+            ok = (item == -1);
+            break;
+        }
         int blk, bh, n_a, n_b;
-        if (!wk.get(p, &blk, &bh, &n_a, &n_b)) continue;
+        wk.get(item, &blk, &bh, &n_a, &n_b);
         const int n_t[2] = {n_a, n_b};
         const int n = max(n_a, n_b);
         const int qs = w % Cfg::kQStages;
 #pragma unroll
         for (int t = 0; t < 2; ++t)
             q_k[t] = umma_desc_lo(smem_u32(smem + Cfg::kOffQ + (qs * 2 + t) * Cfg::kTileBytes), 16);
-        ok = mbar_wait(&bars->q_full[qs], (w / Cfg::kQStages) & 1, abort_flag, limit);
-        if (ok) ok = mbar_wait(&bars->k_full[g & 1], (g >> 1) & 1, abort_flag, limit);
-        if (!ok) break;
-        tc_fence_after();
-        // P over S: the S columns of both tiles are free, their last P was consumed by a P V queued
-        // earlier.  P apart: issue_qk waits until the previous S_t has been read.
-        if (n_a > 0) issue_qk(0, g);
-        if (n_b > 0 && ok) issue_qk(1, g);
-        if (!ok) break;
-        if (el) tc_commit(&bars->k_empty[g & 1]);  // K tile 0 is no longer read once these have run
-        __syncwarp();
+        if (!first_queued) {
+            ok = mbar_wait(&bars->q_full[qs], (w / Cfg::kQStages) & 1, abort_flag, limit);
+            if (ok) ok = mbar_wait(&bars->k_full[g & 1], (g >> 1) & 1, abort_flag, limit);
+            if (!ok) break;
+            tc_fence_after();
+            // P over S: the S columns of both tiles are free, their last P was consumed by a P V queued
+            // earlier.  P apart: issue_qk waits until the previous S_t has been read.
+            if (n_a > 0) issue_qk(0, g, q_k[0]);
+            if (n_b > 0 && ok) issue_qk(1, g, q_k[1]);
+            if (!ok) break;
+            if (el) tc_commit(&bars->k_empty[g & 1]);  // K tile 0 is no longer read once these have run
+            __syncwarp();
+        }
+        first_queued = false;
         for (int j = 0; j < n && ok; ++j, ++g) {
             const int st = g & 1;
             bool next_k_ready = false;
@@ -226,8 +273,37 @@ __device__ __forceinline__ void fwd_mma(uint8_t* smem, FwdBars* bars, uint32_t t
                 tc_fence_after();
 #pragma unroll
                 for (int t = 0; t < 2; ++t)
-                    if (j + 1 < n_t[t] && ok) issue_qk(t, g + 1);
+                    if (j + 1 < n_t[t] && ok) issue_qk(t, g + 1, q_k[t]);
                 if (!ok) break;
+            } else if (Cfg::kSepP && Cfg::kQStages > 1) {
+                // Last key tile of the item: if the producer has already announced the next item and its Q
+                // tiles and first K tile have landed, its first Q K^T products are queued now, exactly like
+                // those of a next key tile, so that neither softmax warpgroup waits at the item boundary.
+                const int wn = w + 1;
+                bool there = mbar_try_wait(&bars->work_full[wn & 1], (wn >> 1) & 1);
+                if (__all_sync(0xffffffffu, there)) {
+                    peeked = *reinterpret_cast<volatile int*>(&bars->work_item[wn & 1]);
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&bars->work_empty[wn & 1]);
+                    if (peeked >= 0) {
+                        const int qs2 = wn % Cfg::kQStages;
+                        there = mbar_try_wait(&bars->q_full[qs2], (wn / Cfg::kQStages) & 1) &&
+                                mbar_try_wait(&bars->k_full[st ^ 1], ((g + 1) >> 1) & 1);
+                        if (__all_sync(0xffffffffu, there)) {
+                            int blk2, bh2, n_a2, n_b2;
+                            wk.get(peeked, &blk2, &bh2, &n_a2, &n_b2);
+                            tc_fence_after();
+                            if (n_a2 > 0)
+                                issue_qk(0, g + 1, umma_desc_lo(smem_u32(smem + Cfg::kOffQ + (qs2 * 2 + 0) * Cfg::kTileBytes), 16));
+                            if (n_b2 > 0 && ok)
+                                issue_qk(1, g + 1, umma_desc_lo(smem_u32(smem + Cfg::kOffQ + (qs2 * 2 + 1) * Cfg::kTileBytes), 16));
+                            if (!ok) break;
+                            if (el) tc_commit(&bars->k_empty[st ^ 1]);
+                            __syncwarp();
+                            first_queued = true;
+                        }
+                    }
+                }
             }
 #pragma unroll
             for (int t = 0; t < 2; ++t) {
@@ -263,7 +339,7 @@ __device__ __forceinline__ void fwd_mma(uint8_t* smem, FwdBars* bars, uint32_t t
                         tc_fence_after();
                         next_k_ready = true;
                     }
-                    issue_qk(t, g + 1);
+                    issue_qk(t, g + 1, q_k[t]);
                 }
             }
             if (!ok) break;
@@ -273,6 +349,7 @@ __device__ __forceinline__ void fwd_mma(uint8_t* smem, FwdBars* bars, uint32_t t
             }
             __syncwarp();
         }
+        if (!ok) break;
         if (n_a > 0) ++wt[0];
         if (n_b > 0) ++wt[1];
         ++w;
@@ -303,9 +380,14 @@ __device__ __forceinline__ void fwd_softmax(uint8_t* smem, FwdBars* bars, uint32
     bool ok = true;
     int w = 0, wt = 0, cnt = 0;  // items, items this tile took part in, key tiles processed by this tile
 
-    for (int p = 0; p < wk.passes() && ok; ++p) {
+    for (;;) {
+        const int item = next_item(bars, w, lane, limit);
+        if (item < 0) {
+            ok = (item == -1);
+            break;
+        }
         int blk, bh, n_a, n_b;
-        if (!wk.get(p, &blk, &bh, &n_a, &n_b)) continue;
+        wk.get(item, &blk, &bh, &n_a, &n_b);
         const int n_kv = (t == 0) ? n_a : n_b;
         const int qt = 2 * blk + t;
         const int row = qt * kBlockQ + row_local;
@@ -320,6 +402,7 @@ __device__ __forceinline__ void fwd_softmax(uint8_t* smem, FwdBars* bars, uint32
                 if (leader_ok) mbar_arrive(&bars->q_empty[qs]);
             }
             ok = __all_sync(0xffffffffu, leader_ok);
+            if (!ok) break;
             ++w;
             continue;
         }
@@ -476,6 +559,7 @@ __device__ __forceinline__ void fwd_softmax(uint8_t* smem, FwdBars* bars, uint32
         // Brings the leader back together with the rest of its warp before the next warp-wide TMEM
         // load, and makes a failed wait of the leader a failure of the whole warp.
         ok = __all_sync(0xffffffffu, leader_ok);
+        if (!ok) break;
         ++w;
         ++wt;
     }
@@ -493,8 +577,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     FwdBars* bars = reinterpret_cast<FwdBars*>(smem + Cfg::kOffBar);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const FwdWork wk{n_blocks * BH, static_cast<int>(gridDim.x), static_cast<int>(blockIdx.x), BH, n_blocks,
-                     (T + kBlockK - 1) / kBlockK, T, H, orders, kCausal};
+    const FwdWork wk{n_blocks * BH, BH, n_blocks, (T + kBlockK - 1) / kBlockK, T, H, orders, kCausal};
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < 2; ++s) {
@@ -512,6 +595,11 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             mbar_init(&bars->o_staged[s], 4);
         }
         mbar_init(&bars->drain, 1);
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(&bars->work_full[s], 1);
+            mbar_init(&bars->work_empty[s], kWorkConsumers);
+        }
+        mbar_init(&bars->clc_bar, 1);
         bars->abort_flag = 0;
         fence_mbar_init();
         tma_prefetch_desc(&tmQ);
@@ -530,7 +618,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     griddep_launch_dependents();
     if (warp == 0 && lane == 0) {  // the first item's Q tiles and first K, V tiles on their way into L2 meanwhile
         int blk, bh, n_a, n_b;
-        if (wk.get(0, &blk, &bh, &n_a, &n_b)) {
+        {
+            wk.get(blockIdx.x, &blk, &bh, &n_a, &n_b);
             const int head = kStrided ? bh % wk.H : 0, batch = kStrided ? bh / wk.H : 0;
 #pragma unroll
             for (int h = 0; h < Cfg::kHalves; ++h) {
@@ -565,7 +654,8 @@ cudaError_t launch_one(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUt
     const int n_blocks = (s.T + kBlockRows - 1) / kBlockRows;
     const int BH = s.B * s.H;
     const long long n_items = static_cast<long long>(n_blocks) * BH;
-    const dim3 grid(static_cast<unsigned>(n_items < num_sms ? n_items : num_sms));  // one persistent CTA per SM
+    (void)num_sms;
+    const dim3 grid(static_cast<unsigned>(n_items));  // one CTA per item; those that do not start at once are taken over
     if (strided)
         return launch_overlapped(attn_fwd_kernel<D, kCausal, true>, grid, dim3(kFwdThreads), FwdCfg<D>::kSmemBytes,
                                  stream, tmQ, tmK, tmV, tmO, LSE, s.T, BH, s.H, orders, n_blocks, s.scale, wait_limit, inject, dev_status);

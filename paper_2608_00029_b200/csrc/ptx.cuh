@@ -112,6 +112,35 @@ __device__ __forceinline__ bool mbar_wait_relaxed(uint64_t* bar, uint32_t parity
     }
 }
 
+// ------------------------------------------------------------------ dynamic work distribution
+// A persistent CTA that has finished its work item asks the hardware to cancel the launch of a CTA of the same
+// grid that has not started yet and takes over that CTA's index (sm_100 cluster launch control).  The grid is
+// launched with one CTA per work item; as many as fit start at once, the rest are handed out this way in
+// launch order, so that no CTA idles while another still has items queued.  The request is asynchronous: the
+// 16-byte answer lands in shared memory and completes 16 bytes on `bar`.  After a request has failed (nothing
+// left to cancel) no further request may be made.
+__device__ __forceinline__ void clc_try_cancel(void* smem_response16, uint64_t* bar) {
+    asm volatile(
+        "clusterlaunchcontrol.try_cancel.async.shared::cta.mbarrier::complete_tx::bytes.b128 [%0], [%1];"
+        ::"r"(smem_u32(smem_response16)), "r"(smem_u32(bar))
+        : "memory");
+}
+// Decodes an answer: the x index of the cancelled CTA, or -1 if nothing was cancelled.
+__device__ __forceinline__ int clc_cancelled_cta(const void* smem_response16) {
+    uint32_t ok, x;
+    asm volatile(
+        "{\n\t.reg .b128 r;\n\t.reg .pred p;\n\t"
+        "ld.shared.b128 r, [%2];\n\t"
+        "clusterlaunchcontrol.query_cancel.is_canceled.pred.b128 p, r;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t"
+        "mov.u32 %1, 0;\n\t"
+        "@p clusterlaunchcontrol.query_cancel.get_first_ctaid::x.b32.b128 %1, r;\n\t}"
+        : "=r"(ok), "=r"(x)
+        : "r"(smem_u32(smem_response16))
+        : "memory");
+    return ok ? static_cast<int>(x) : -1;
+}
+
 // ------------------------------------------------------------------------------------------ TMA
 __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* m) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(m) : "memory");

@@ -68,6 +68,8 @@ def test_device_arm_line(launch):
         assert t[leg]["ms"] > 0 and abs(t[leg]["frac"] - t[leg]["tflops"] / r["peak"]) < 1e-9
     k = r["kernel_ms"]
     assert t["bwd"]["ms"] > k["bwd_main"] * 0.9   # the sequence contains the main kernel
+    assert set(r["kernel_ms_eager"]) == set(k) and "graph" in r["attribution"]
+    assert all(k[n] <= r["kernel_ms_eager"][n] * 1.1 for n in k)   # back to back is never slower than with host gaps
     e = d["e2e"]
     assert e["h2d_bytes_per_step"] == e["d2h_bytes_per_step"] == 4 * 8 * 12 * 1024 * 64 * 2
     assert 0 < e["value"] < d["value"]  # the copies are inside the timed region
