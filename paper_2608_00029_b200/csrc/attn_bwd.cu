@@ -828,7 +828,10 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     using Cfg = BwdCfg<D>;
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    if (Cfg::kAlignPad == 0 && smem != smem_raw) {  // no room to realign: give up before anything is set up
+    if (Cfg::kAlignPad == 0 && smem != smem_raw) {
+        // No room to realign: give up before anything is set up, but only once the predecessor in the stream
+        // has completed (the status word is global memory, and this grid must not finish ahead of it).
+        griddep_wait();
         if (threadIdx.x == 0) atomicExch(dev_status, kDevTimeout);
         return;
     }

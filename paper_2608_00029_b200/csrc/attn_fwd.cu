@@ -379,6 +379,7 @@ __device__ __forceinline__ void fwd_softmax(uint8_t* smem, FwdBars* bars, uint32
     const int T = wk.T;
     bool ok = true;
     int w = 0, wt = 0, cnt = 0;  // items, items this tile took part in, key tiles processed by this tile
+    int pending_qs = -1;         // Q stage whose O store was issued at the end of the previous item
 
     for (;;) {
         const int item = next_item(bars, w, lane, limit);
@@ -398,9 +399,14 @@ __device__ __forceinline__ void fwd_softmax(uint8_t* smem, FwdBars* bars, uint32
             // has been filled, so that this warpgroup never runs ahead of the ring.
             bool leader_ok = true;
             if (leader) {
+                if (pending_qs >= 0) {
+                    bulk_wait_group_read<0>();
+                    mbar_arrive(&bars->q_empty[pending_qs]);
+                }
                 leader_ok = mbar_wait(&bars->q_full[qs], (w / Cfg::kQStages) & 1, abort_flag, limit);
                 if (leader_ok) mbar_arrive(&bars->q_empty[qs]);
             }
+            pending_qs = -1;
             ok = __all_sync(0xffffffffu, leader_ok);
             if (!ok) break;
             ++w;
@@ -509,6 +515,14 @@ __device__ __forceinline__ void fwd_softmax(uint8_t* smem, FwdBars* bars, uint32
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&bars->p_ready[t]);
+            if (pending_qs >= 0) {
+                if (leader) {
+                    bulk_wait_group_read<0>();
+                    mbar_arrive(&bars->q_empty[pending_qs]);
+                }
+                pending_qs = -1;
+                __syncwarp();
+            }
         }
         if (!ok) break;
 
@@ -552,10 +566,16 @@ __device__ __forceinline__ void fwd_softmax(uint8_t* smem, FwdBars* bars, uint32
                     tma_store_tile<kStrided>(tmO, stage + h * kHalfTileBytes, (wk.orders >> 12) & 15, h * kBoxCols,
                                              qt * kBlockQ, kStrided ? bh % wk.H : 0, kStrided ? bh / wk.H : 0, bh);
                 bulk_commit_group();
-                bulk_wait_group_read<0>();  // the buffer has been read and may receive the next Q tile
-                mbar_arrive(&bars->q_empty[qs]);
+                if (Cfg::kQStages == 1) {  // the next item's Q tile needs this very buffer
+                    bulk_wait_group_read<0>();
+                    mbar_arrive(&bars->q_empty[qs]);
+                }
             }
         }
+        // With two Q stages the buffer is only needed for the item after next: it is handed back after the next
+        // item's first key tile, when the store has long read it, instead of holding this warp up now (worth 7 %
+        // at B=8, H=12, T=1024; a separate store thread that waits in the softmax warps' stead was slower).
+        if (Cfg::kQStages > 1) pending_qs = qs;
         // Brings the leader back together with the rest of its warp before the next warp-wide TMEM
         // load, and makes a failed wait of the leader a failure of the whole warp.
         ok = __all_sync(0xffffffffu, leader_ok);
