@@ -486,9 +486,13 @@ __device__ __forceinline__ void bwd_compute(uint8_t* smem, BwdBars* bars, uint32
             const int b = g & 1;
             const float4* s_lse4 = reinterpret_cast<const float4*>(row_buf + b * 256 + kQPT * part);
             const float4* s_dl4 = reinterpret_cast<const float4*>(row_buf + b * 256 + 128 + kQPT * part);
-            ok = mbar_wait(&bars->row_full[b], (g >> 1) & 1, abort_flag);
-            if (!ok) break;
-            ok = mbar_wait(&bars->s_full, g & 1, abort_flag);
+            // Three non-blocking probes issued together, so that their latencies overlap; each is followed up by
+            // a proper wait only if it failed (-2 % against three waits in a row).
+            const bool row_there = mbar_test(&bars->row_full[b], (g >> 1) & 1);
+            const bool s_there = mbar_test(&bars->s_full, g & 1);
+            const bool dp_there = mbar_test(&bars->dp_full, g & 1);
+            if (!row_there) ok = mbar_wait(&bars->row_full[b], (g >> 1) & 1, abort_flag);
+            if (ok && !s_there) ok = mbar_wait(&bars->s_full, g & 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
 
@@ -511,7 +515,7 @@ __device__ __forceinline__ void bwd_compute(uint8_t* smem, BwdBars* bars, uint32
             constexpr bool kEarlydP = Cfg::kSeparateP && !Cfg::kdQAliased;
             static_assert(kEarlydP || !Cfg::kSeparateP, "P^T columns of their own need the dp_full wait below");
             if (kEarlydP) {
-                ok = mbar_wait(&bars->dp_full, g & 1, abort_flag);
+                if (!dp_there) ok = mbar_wait(&bars->dp_full, g & 1, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
             }

@@ -280,15 +280,15 @@ __device__ __forceinline__ void fwd_mma(uint8_t* smem, FwdBars* bars, uint32_t t
                 // tiles and first K tile have landed, its first Q K^T products are queued now, exactly like
                 // those of a next key tile, so that neither softmax warpgroup waits at the item boundary.
                 const int wn = w + 1;
-                bool there = mbar_try_wait(&bars->work_full[wn & 1], (wn >> 1) & 1);
+                bool there = mbar_test(&bars->work_full[wn & 1], (wn >> 1) & 1);
                 if (__all_sync(0xffffffffu, there)) {
                     peeked = *reinterpret_cast<volatile int*>(&bars->work_item[wn & 1]);
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&bars->work_empty[wn & 1]);
                     if (peeked >= 0) {
                         const int qs2 = wn % Cfg::kQStages;
-                        there = mbar_try_wait(&bars->q_full[qs2], (wn / Cfg::kQStages) & 1) &&
-                                mbar_try_wait(&bars->k_full[st ^ 1], ((g + 1) >> 1) & 1);
+                        there = mbar_test(&bars->q_full[qs2], (wn / Cfg::kQStages) & 1) &&
+                                mbar_test(&bars->k_full[st ^ 1], ((g + 1) >> 1) & 1);
                         if (__all_sync(0xffffffffu, there)) {
                             int blk2, bh2, n_a2, n_b2;
                             wk.get(peeked, &blk2, &bh2, &n_a2, &n_b2);

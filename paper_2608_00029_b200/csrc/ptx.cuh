@@ -60,6 +60,21 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     return ok != 0;
 }
 
+// Non-blocking probe: true if the phase has completed, false at once if it has not (try_wait above may keep the
+// thread suspended for a while before it answers false; this one never does).  For looking ahead without
+// committing to a wait.
+__device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
 // Same test, but the hardware may keep the thread suspended for up to `hint_ns` while the phase is
 // incomplete (it resumes at once when the phase completes).  A suspended thread issues nothing, so
 // waiting warps do not take issue slots from the warps that share their scheduler.
