@@ -62,10 +62,7 @@ struct FwdBars {
     uint64_t k_full[2], k_empty[2], v_full[2], v_empty[2];
     uint64_t s_full[2], s_free[2], p_ready[2], pv_done[2], o_free[2], o_staged[2];  // per query tile
     uint64_t drain;
-    uint64_t work_full[2], work_empty[2];  // ring of item numbers: producer -> UMMA issuer and softmax warps
-    uint64_t clc_bar;                      // the answer to a cancellation request has arrived
-    uint4 clc_response;
-    int work_item[2];
+    WorkRing ring;  // item numbers: producer -> UMMA issuer and softmax warps
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -88,16 +85,6 @@ struct FwdWork {
     }
 };
 
-// Consumer side of the item ring: the number of the w-th item of this CTA, -1 when there are no more, -2 if
-// the wait was given up.  Every lane of the calling warp gets the same answer.
-__device__ __forceinline__ int next_item(FwdBars* bars, int w, int lane, long long limit) {
-    if (!mbar_wait(&bars->work_full[w & 1], (w >> 1) & 1, &bars->abort_flag, limit)) return -2;
-    const int item = *reinterpret_cast<volatile int*>(&bars->work_item[w & 1]);
-    __syncwarp();
-    if (lane == 0) mbar_arrive(&bars->work_empty[w & 1]);
-    return item;
-}
-
 template <int D, bool kStrided>
 __device__ __forceinline__ void fwd_producer(const CUtensorMap* tmQ, const CUtensorMap* tmK,
                                              const CUtensorMap* tmV, uint8_t* smem, FwdBars* bars,
@@ -111,11 +98,8 @@ __device__ __forceinline__ void fwd_producer(const CUtensorMap* tmQ, const CUten
     bool clc_pending = false;
     for (;;) {
         // hand the item (or the end mark) to the other roles
-        ok = mbar_wait(&bars->work_empty[w & 1], ((w >> 1) & 1) ^ 1, abort_flag, limit);
-        if (!ok) break;
-        bars->work_item[w & 1] = item;
-        mbar_arrive(&bars->work_full[w & 1]);
-        if (item < 0) break;
+        ok = bars->ring.publish(w, item, abort_flag, limit);
+        if (!ok || item < 0) break;
         int blk, bh, n_a, n_b;
         wk.get(item, &blk, &bh, &n_a, &n_b);
         const int head = kStrided ? bh % wk.H : 0, batch = kStrided ? bh / wk.H : 0;
@@ -161,19 +145,17 @@ __device__ __forceinline__ void fwd_producer(const CUtensorMap* tmQ, const CUten
         // All loads of this item are on their way (the other roles are about two key tiles behind): only now
         // ask for the next item, so that an item is claimed as late as possible and the CTAs that finish early
         // find the remaining ones.
-        mbar_expect_tx(&bars->clc_bar, 16);
-        clc_try_cancel(&bars->clc_response, &bars->clc_bar);
+        bars->ring.request();
         clc_pending = true;
-        ok = mbar_wait(&bars->clc_bar, w & 1, abort_flag, limit);
+        ok = bars->ring.answer(w, &item, abort_flag, limit);
         if (!ok) break;
         clc_pending = false;
-        item = clc_cancelled_cta(&bars->clc_response);
         ++w;
     }
     if (!ok) {
         // Giving up: let the copies already in flight land before the CTA's shared memory goes away.
         int none = 0;
-        if (clc_pending) (void)mbar_wait(&bars->clc_bar, w & 1, &none);  // the answer must land before the CTA ends
+        if (clc_pending) (void)mbar_wait(&bars->ring.answer_bar, w & 1, &none);  // the answer must land before the CTA ends
         for (int s = 0; s < 2; ++s) {
             if (armed_q[s] >= 0) (void)mbar_wait(&bars->q_full[s], armed_q[s], &none);
             if (armed_k[s] >= 0) (void)mbar_wait(&bars->k_full[s], armed_k[s], &none);
@@ -234,7 +216,7 @@ __device__ __forceinline__ void fwd_mma(uint8_t* smem, FwdBars* bars, uint32_t t
     int peeked = kNotPeeked;  // the next item's number, if it was looked at from inside the current item
     bool first_queued = false;  // ... and its first Q K^T products were queued from there
     for (;;) {
-        const int item = (peeked != kNotPeeked) ? peeked : next_item(bars, w, lane, limit);
+        const int item = (peeked != kNotPeeked) ? peeked : bars->ring.take(w, lane, abort_flag, limit);
         peeked = kNotPeeked;
         if (item < 0) {
             ok = (item == -1);
@@ -280,14 +262,11 @@ __device__ __forceinline__ void fwd_mma(uint8_t* smem, FwdBars* bars, uint32_t t
                 // tiles and first K tile have landed, its first Q K^T products are queued now, exactly like
                 // those of a next key tile, so that neither softmax warpgroup waits at the item boundary.
                 const int wn = w + 1;
-                bool there = mbar_test(&bars->work_full[wn & 1], (wn >> 1) & 1);
-                if (__all_sync(0xffffffffu, there)) {
-                    peeked = *reinterpret_cast<volatile int*>(&bars->work_item[wn & 1]);
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&bars->work_empty[wn & 1]);
+                if (bars->ring.published(wn)) {
+                    peeked = bars->ring.take(wn, lane, abort_flag, limit);
                     if (peeked >= 0) {
                         const int qs2 = wn % Cfg::kQStages;
-                        there = mbar_test(&bars->q_full[qs2], (wn / Cfg::kQStages) & 1) &&
+                        bool there = mbar_test(&bars->q_full[qs2], (wn / Cfg::kQStages) & 1) &&
                                 mbar_test(&bars->k_full[st ^ 1], ((g + 1) >> 1) & 1);
                         if (__all_sync(0xffffffffu, there)) {
                             int blk2, bh2, n_a2, n_b2;
@@ -382,7 +361,7 @@ __device__ __forceinline__ void fwd_softmax(uint8_t* smem, FwdBars* bars, uint32
     int pending_qs = -1;         // Q stage whose O store was issued at the end of the previous item
 
     for (;;) {
-        const int item = next_item(bars, w, lane, limit);
+        const int item = bars->ring.take(w, lane, abort_flag, limit);
         if (item < 0) {
             ok = (item == -1);
             break;
@@ -615,11 +594,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             mbar_init(&bars->o_staged[s], 4);
         }
         mbar_init(&bars->drain, 1);
-        for (int s = 0; s < 2; ++s) {
-            mbar_init(&bars->work_full[s], 1);
-            mbar_init(&bars->work_empty[s], kWorkConsumers);
-        }
-        mbar_init(&bars->clc_bar, 1);
+        bars->ring.init(kWorkConsumers);
         bars->abort_flag = 0;
         fence_mbar_init();
         tma_prefetch_desc(&tmQ);

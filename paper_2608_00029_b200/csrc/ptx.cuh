@@ -156,6 +156,59 @@ __device__ __forceinline__ int clc_cancelled_cta(const void* smem_response16) {
     return ok ? static_cast<int>(x) : -1;
 }
 
+// The ring through which a CTA's producer thread tells the other roles which work item comes next: two
+// entries in shared memory.  The producer publishes the number of the w-th item of this CTA (or -1: no more),
+// each consumer warp (or single-thread role) takes it and frees the entry.  The producer gets the numbers
+// from the hardware: its own CTA index first, then the indices of CTAs whose launch it cancels.
+struct WorkRing {
+    uint64_t full[2], empty[2], answer_bar;
+    uint4 response;
+    int item[2];
+
+    __device__ __forceinline__ void init(int consumers) {
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(&full[s], 1);
+            mbar_init(&empty[s], consumers);
+        }
+        mbar_init(&answer_bar, 1);
+    }
+    // ---- producer (one thread)
+    __device__ __forceinline__ bool publish(int w, int it, volatile int* abort_flag, long long limit) {
+        if (!mbar_wait(&empty[w & 1], ((w >> 1) & 1) ^ 1, abort_flag, limit)) return false;
+        item[w & 1] = it;
+        mbar_arrive(&full[w & 1]);
+        return true;
+    }
+    // Asks for the item after the w-th; at most one request is outstanding, and none follows a failed one.
+    __device__ __forceinline__ void request() {
+        mbar_expect_tx(&answer_bar, 16);
+        clc_try_cancel(&response, &answer_bar);
+    }
+    __device__ __forceinline__ bool answer(int w, int* next, volatile int* abort_flag, long long limit) {
+        if (!mbar_wait(&answer_bar, w & 1, abort_flag, limit)) return false;
+        *next = clc_cancelled_cta(&response);
+        return true;
+    }
+    // ---- consumers: the w-th item, -1 when there are no more, -2 if the wait was given up
+    __device__ __forceinline__ int take(int w, int lane, volatile int* abort_flag, long long limit) {  // a whole warp
+        if (!mbar_wait(&full[w & 1], (w >> 1) & 1, abort_flag, limit)) return -2;
+        const int it = *reinterpret_cast<volatile int*>(&item[w & 1]);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&empty[w & 1]);
+        return it;
+    }
+    __device__ __forceinline__ int take_single(int w, volatile int* abort_flag, long long limit) {  // one thread
+        if (!mbar_wait(&full[w & 1], (w >> 1) & 1, abort_flag, limit)) return -2;
+        const int it = *reinterpret_cast<volatile int*>(&item[w & 1]);
+        mbar_arrive(&empty[w & 1]);
+        return it;
+    }
+    // Has the w-th item been published yet?  Non-blocking; the same answer in every lane of a converged warp.
+    __device__ __forceinline__ bool published(int w) {
+        return __all_sync(0xffffffffu, mbar_test(&full[w & 1], (w >> 1) & 1));
+    }
+};
+
 // ------------------------------------------------------------------------------------------ TMA
 __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* m) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(m) : "memory");
