@@ -245,6 +245,21 @@ int nova_attn_last_cuda_error(void);
 int nova_attn_test_configure_waits(long long limit_cycles, int inject);
 
 /*
+ * Host-side view of the backward kernel's work distribution (no GPU is touched): the work items of CTA
+ * `cta` out of `n_ctas` for a problem of B*H = `BH` heads, `T` tokens, head dimension `D`, in the order the
+ * CTA processes them.  An item is one 128-key tile of one head (paper Section 4.2: the backward pass loops
+ * over key tiles and, for each, over the query tiles at or below the diagonal); the list is what decides
+ * load balance and which heads' accumulators are in flight together.  Writes up to `capacity` pairs
+ * (key tile, head index) into `items` (host, 2 * capacity ints; may be NULL when capacity is 0) and the
+ * plan {heads per chunk, chunks, passes per full chunk, passes of the last chunk} into `plan4` (host, 4
+ * ints, may be NULL).  Returns the number of items of that CTA (which may exceed `capacity`), or
+ * NOVA_ATTN_ERR_SHAPE (negative, like every error code) for arguments out of range (BH, T < 1; D not 64 or 128; n_ctas < 1; cta outside
+ * [0, n_ctas)).
+ */
+int nova_attn_bwd_work_list(int BH, long long T, int D, int causal, int n_ctas, int cta, int* items, int capacity,
+                            int* plan4);
+
+/*
  * Synchronises `stream`, then reads and clears the device status word of the current device.
  * Returns NOVA_ATTN_OK, NOVA_ATTN_ERR_TIMEOUT (a kernel gave up on a bounded wait; its outputs are
  * invalid) or NOVA_ATTN_ERR_CUDA.

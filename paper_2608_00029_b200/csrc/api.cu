@@ -13,6 +13,7 @@
 #include "../../include/nova_attn.h"
 #include "../../include/nova_lmhead.h"
 #include "kernels.h"
+#include "work_plan.h"
 
 namespace nova {
 
@@ -545,6 +546,35 @@ int nova_attn_test_configure_waits(long long limit_cycles, int inject) {
     g_wait_limit.store(limit_cycles == 0 ? kDefaultWaitLimit : limit_cycles, std::memory_order_relaxed);
     g_inject.store(inject, std::memory_order_relaxed);
     return NOVA_ATTN_OK;
+}
+
+int nova_attn_bwd_work_list(int BH, long long T, int D, int causal, int n_ctas, int cta, int* items, int capacity,
+                            int* plan4) {
+    if (BH < 1 || T < 1 || (D != 64 && D != 128) || n_ctas < 1 || cta < 0 || cta >= n_ctas || capacity < 0 ||
+        (capacity > 0 && items == nullptr))
+        return NOVA_ATTN_ERR_SHAPE;
+    int n_tiles = 0, grid = 0;
+    const WorkPlan plan = bwd_work_plan(BH, T, D, causal != 0, n_ctas, &n_tiles, &grid);
+    if (plan4 != nullptr) {
+        plan4[0] = plan.chunk;
+        plan4[1] = plan.n_chunks;
+        plan4[2] = plan.passes_per_chunk;
+        plan4[3] = plan.passes_last;
+    }
+    if (cta >= grid) return 0;  // fewer items than CTAs: the grid is that much smaller
+    const WorkArgs wa{BH, n_tiles, 1, 0u, 0, plan};
+    const WorkList wl{wa, causal != 0};
+    int n = 0;
+    for (WorkCursor cur; !wl.done(cur); wl.advance(cur)) {
+        int kt, bh, i0, n_it;
+        if (!wl.get_for(cur, grid, cta, &kt, &bh, &i0, &n_it)) continue;
+        if (n < capacity) {
+            items[2 * n] = kt;
+            items[2 * n + 1] = bh;
+        }
+        ++n;
+    }
+    return n;
 }
 
 int nova_attn_poll_device_status(void* stream) {

@@ -41,6 +41,7 @@
 // one lane does extra work (the dQ leader), the warp is rejoined with a vote before the next one.
 #include "kernels.h"
 #include "ptx.cuh"
+#include "work_plan.h"
 
 namespace nova {
 namespace {
@@ -81,6 +82,11 @@ struct BwdCfg {
     static constexpr int kColdK = 256 + D;
     static constexpr bool kdQAliased = (D == 128);  // dQ reuses the dP^T region
     static constexpr int kColdQ = (D == 64) ? 384 : 128;
+    // Where dQ lies over dP^T, a bf16 dS^T kept in those columns would force dK (which reads it) to run before
+    // dQ (which overwrites it), and dQ, its read-out and the next dP^T are the chain that sets the period of a
+    // tile.  There dK reads dS^T from the shared-memory copy that dQ uses as well (K-major for dK, M-major for
+    // dQ), dQ is queued first and dK runs while the dQ warps empty the columns.
+    static constexpr bool kdKFromSmem = kdQAliased;
     static constexpr bool kSeparateP = (D == 64);   // P^T in its own columns instead of over S^T
     static constexpr int kColP = kSeparateP ? 448 : 0;
     static constexpr int kPHalfStride = kSeparateP ? 32 : 64;  // column distance between the two query halves of P^T
@@ -107,26 +113,6 @@ struct BwdBars {
     int abort_flag;
 };
 
-// This CTA's list of work items.  Items are ordered by weight (key tile 0 of a causal problem sees
-// every query tile, the last key tile only one) and dealt to the CTAs in zig-zag passes.
-struct WorkList {
-    int n_items, n_ctas, cta, BH, n_tiles, H;
-    uint32_t orders;  // coordinate orders of the Q, K, V, dO, dK, dV tensor maps, four bits each
-    bool no_dq;       // dK/dV half of the two-kernel backward: no dQ product, no accumulator traffic
-    bool causal;
-    __device__ __forceinline__ int passes() const { return (n_items + n_ctas - 1) / n_ctas; }
-    // Item of pass p: returns false if this CTA has none in that pass.
-    __device__ __forceinline__ bool get(int p, int* kt, int* bh, int* i0, int* n_it) const {
-        const int idx = p * n_ctas + ((p & 1) ? (n_ctas - 1 - cta) : cta);
-        if (idx >= n_items) return false;
-        *kt = idx / BH;
-        *bh = idx % BH;
-        *i0 = causal ? *kt : 0;  // raised lower bound of the query loop
-        *n_it = n_tiles - *i0;
-        return true;
-    }
-};
-
 template <int D, bool kStrided>
 __device__ __forceinline__ void bwd_producer(const CUtensorMap* tmQ, const CUtensorMap* tmK, const CUtensorMap* tmV,
                                              const CUtensorMap* tmdO, uint8_t* smem, BwdBars* bars,
@@ -136,10 +122,10 @@ __device__ __forceinline__ void bwd_producer(const CUtensorMap* tmQ, const CUten
     int armed_kv[2] = {-1, -1}, armed_q[3] = {-1, -1, -1}, armed_do[2] = {-1, -1};
     bool ok = true;
     int w = 0, g = 0;  // items and query tiles processed so far by this CTA
-    for (int p = 0; p < wl.passes() && ok; ++p) {
+    for (WorkCursor cur; !wl.done(cur) && ok; wl.advance(cur)) {
         int kt, bh, i0, n_it;
-        if (!wl.get(p, &kt, &bh, &i0, &n_it)) continue;
-        const int head = kStrided ? bh % wl.H : 0, batch = kStrided ? bh / wl.H : 0;
+        if (!wl.get(cur, &kt, &bh, &i0, &n_it)) continue;
+        const int head = kStrided ? bh % wl.H() : 0, batch = kStrided ? bh / wl.H() : 0;
         const int ks = w % Cfg::kKVStages;
         const uint32_t kph = (w / Cfg::kKVStages) & 1;
         ok = mbar_wait(&bars->kv_empty[ks], kph ^ 1, abort_flag);
@@ -149,9 +135,9 @@ __device__ __forceinline__ void bwd_producer(const CUtensorMap* tmQ, const CUten
 #pragma unroll
         for (int h = 0; h < Cfg::kHalves; ++h) {
             tma_load_tile<kStrided>(smem + Cfg::kOffK + ks * Cfg::kTileBytes + h * kHalfTileBytes, tmK, &bars->kv_full[ks],
-                          (wl.orders >> 4) & 15, h * kBoxCols, kt * kBlockK, head, batch, bh);
+                          (wl.orders() >> 4) & 15, h * kBoxCols, kt * kBlockK, head, batch, bh);
             tma_load_tile<kStrided>(smem + Cfg::kOffV + ks * Cfg::kTileBytes + h * kHalfTileBytes, tmV, &bars->kv_full[ks],
-                          (wl.orders >> 8) & 15, h * kBoxCols, kt * kBlockK, head, batch, bh);
+                          (wl.orders() >> 8) & 15, h * kBoxCols, kt * kBlockK, head, batch, bh);
         }
         for (int it = 0; it < n_it; ++it, ++g) {
             const int st = g % Cfg::kQStages;
@@ -163,7 +149,7 @@ __device__ __forceinline__ void bwd_producer(const CUtensorMap* tmQ, const CUten
 #pragma unroll
             for (int h = 0; h < Cfg::kHalves; ++h)
                 tma_load_tile<kStrided>(smem + Cfg::kOffQ + st * Cfg::kTileBytes + h * kHalfTileBytes, tmQ, &bars->q_full[st],
-                              wl.orders & 15, h * kBoxCols, qrow, head, batch, bh);
+                              wl.orders() & 15, h * kBoxCols, qrow, head, batch, bh);
             const int ds = g % Cfg::kdOStages;
             const uint32_t dph = (g / Cfg::kdOStages) & 1;
             ok = mbar_wait(&bars->do_empty[ds], dph ^ 1, abort_flag);
@@ -173,7 +159,7 @@ __device__ __forceinline__ void bwd_producer(const CUtensorMap* tmQ, const CUten
 #pragma unroll
             for (int h = 0; h < Cfg::kHalves; ++h)
                 tma_load_tile<kStrided>(smem + Cfg::kOffdO + ds * Cfg::kTileBytes + h * kHalfTileBytes, tmdO, &bars->do_full[ds],
-                              (wl.orders >> 12) & 15, h * kBoxCols, qrow, head, batch, bh);
+                              (wl.orders() >> 12) & 15, h * kBoxCols, qrow, head, batch, bh);
         }
         ++w;
     }
@@ -196,6 +182,7 @@ __device__ __forceinline__ void bwd_mma(uint8_t* smem, BwdBars* bars, uint32_t t
     constexpr uint32_t kIdescT = umma_idesc_bf16(128, 128, 0, 0);   // S^T, dP^T
     constexpr uint32_t kIdescKV = umma_idesc_bf16(128, D, 0, 1);    // dV, dK (A from TMEM, B MN-major)
     constexpr uint32_t kIdescdQ = umma_idesc_bf16(128, 64, 1, 1);   // dQ half (A M-major smem, B MN-major)
+    constexpr uint32_t kIdescdQWide = umma_idesc_bf16(128, D, 1, 1);  // all D columns of dQ at once
     const uint32_t t_s = tmem_base + Cfg::kColS, t_dp = tmem_base + Cfg::kColdP;
     const uint32_t t_dv = tmem_base + Cfg::kColdV, t_dk = tmem_base + Cfg::kColdK;
     const uint32_t t_p = tmem_base + Cfg::kColP;
@@ -214,6 +201,7 @@ __device__ __forceinline__ void bwd_mma(uint8_t* smem, BwdBars* bars, uint32_t t
         do_m[st] = umma_desc_lo(smem_u32(smem + Cfg::kOffdO + (st % Cfg::kdOStages) * Cfg::kTileBytes), kHalfTileBytes);
     }
     const uint32_t ds_m = umma_desc_lo(smem_u32(smem + Cfg::kOffdS), kHalfTileBytes);
+    const uint32_t ds_k = umma_desc_lo(smem_u32(smem + Cfg::kOffdS), 16);
     uint32_t k_k = 0, v_k = 0, k_m = 0;  // per item
     // The whole warp runs this role in uniform control flow; one elected lane issues.
     const bool el = elect_one();
@@ -246,14 +234,16 @@ __device__ __forceinline__ void bwd_mma(uint8_t* smem, BwdBars* bars, uint32_t t
     bool ok = true;
     bool first_queued = false;  // S^T and dP^T of this item's first tile were queued during the previous item
     int w = 0, g = 0;
-    for (int p = 0; p < wl.passes() && ok; ++p) {
+    for (WorkCursor cur; !wl.done(cur) && ok; wl.advance(cur)) {
         int kt, bh, i0, n_it;
-        if (!wl.get(p, &kt, &bh, &i0, &n_it)) continue;
+        if (!wl.get(cur, &kt, &bh, &i0, &n_it)) continue;
         // With K/V double-buffered the next item's tiles arrive while this one runs, and the products
         // of its first query tile are queued from inside this item's last iteration (below), exactly
         // as for any other next tile: the compute warps never see the item boundary.
         int kt_n, bh_n, i0_n, n_it_n;
-        const bool has_next = Cfg::kKVStages > 1 && p + 1 < wl.passes() && wl.get(p + 1, &kt_n, &bh_n, &i0_n, &n_it_n);
+        WorkCursor nxt = cur;
+        wl.advance(nxt);
+        const bool has_next = Cfg::kKVStages > 1 && !wl.done(nxt) && wl.get(nxt, &kt_n, &bh_n, &i0_n, &n_it_n);
         const int ks_n = (w + 1) % Cfg::kKVStages;
         const uint32_t k_k_n = umma_desc_lo(smem_u32(smem + Cfg::kOffK + ks_n * Cfg::kTileBytes), 16);
         const uint32_t v_k_n = umma_desc_lo(smem_u32(smem + Cfg::kOffV + ks_n * Cfg::kTileBytes), 16);
@@ -263,7 +253,7 @@ __device__ __forceinline__ void bwd_mma(uint8_t* smem, BwdBars* bars, uint32_t t
         v_k = umma_desc_lo(smem_u32(smem + Cfg::kOffV + ks * Cfg::kTileBytes), 16);
         ok = mbar_wait(&bars->kv_full[ks], (w / Cfg::kKVStages) & 1, abort_flag);
         if (ok) ok = mbar_wait(&bars->q_full[g % Cfg::kQStages], (g / Cfg::kQStages) & 1, abort_flag);
-        if (ok && Cfg::kdQAliased && g > 0 && !wl.no_dq) ok = mbar_wait(&bars->dq_free, (g - 1) & 1, abort_flag);
+        if (ok && Cfg::kdQAliased && g > 0 && !wl.no_dq()) ok = mbar_wait(&bars->dq_free, (g - 1) & 1, abort_flag);
         if (ok) ok = mbar_wait(&bars->do_full[g % Cfg::kdOStages], (g / Cfg::kdOStages) & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
@@ -311,6 +301,28 @@ __device__ __forceinline__ void bwd_mma(uint8_t* smem, BwdBars* bars, uint32_t t
             ok = mbar_wait(&bars->ds_ready, g & 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
+            if (Cfg::kdKFromSmem) {
+                // dQ_i = dS K_j first, all D columns per instruction (the dP^T columns it lands in were read by the
+                // compute warps before they arrived on ds_ready), then dK += dS^T Q_i with dS^T from shared memory.
+                if (el) {
+                    if (!wl.no_dq()) {
+#pragma unroll
+                        for (int k = 0; k < kBlockK / 16; ++k)
+                            umma_ss(tmem_base + Cfg::kColdQ, umma_desc_join(ds_m + k * 128, hi),
+                                    umma_desc_join(k_m + k * 128, hi), kIdescdQWide, k > 0 ? 1u : 0u);
+                        tc_commit(&bars->dq_full);
+                    }
+                    const uint32_t b = q_m0 + (g % Cfg::kQStages) * kQStageStep;
+#pragma unroll
+                    for (int k = 0; k < kBlockQ / 16; ++k) {
+                        const uint32_t off = ((k / 4) * kHalfTileBytes + (k % 4) * 32) >> 4;
+                        umma_ss(t_dk, umma_desc_join(ds_k + off, hi), umma_desc_join(b + k * 128, hi), kIdescKV,
+                                (it > 0 || k > 0) ? 1u : 0u);
+                    }
+                    tc_commit(&bars->q_empty[g % Cfg::kQStages]);
+                }
+                __syncwarp();
+            } else {
             if (el) {
                 const uint32_t b = q_m0 + (g % Cfg::kQStages) * kQStageStep;
 #pragma unroll
@@ -323,12 +335,12 @@ __device__ __forceinline__ void bwd_mma(uint8_t* smem, BwdBars* bars, uint32_t t
             }
             __syncwarp();
             // dQ_i = dS K_j, 64 head-dim columns per accumulator half; 16 keys per instruction.
-            if (!Cfg::kdQAliased && !wl.no_dq) {  // the dQ warps must have read the previous tile out of the dQ columns
+            if (!Cfg::kdQAliased && !wl.no_dq()) {  // the dQ warps must have read the previous tile out of the dQ columns
                 ok = mbar_wait(&bars->dq_free, (g & 1) ^ 1, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
             }
-            if (el && !wl.no_dq) {
+            if (el && !wl.no_dq()) {
 #pragma unroll
                 for (int h = 0; h < Cfg::kHalves; ++h) {
                     const uint32_t t_dq = tmem_base + Cfg::kColdQ + h * 64;
@@ -341,8 +353,9 @@ __device__ __forceinline__ void bwd_mma(uint8_t* smem, BwdBars* bars, uint32_t t
                 tc_commit(&bars->dq_full);
             }
             __syncwarp();
+            }
             if (more || cross) {
-                if (Cfg::kdQAliased && !wl.no_dq) {  // dQ sits in the dP^T region until the dQ warps have read it
+                if (Cfg::kdQAliased && !wl.no_dq()) {  // dQ sits in the dP^T region until the dQ warps have read it
                     ok = mbar_wait(&bars->dq_free, g & 1, abort_flag);
                     if (!ok) break;
                 }
@@ -375,9 +388,9 @@ __device__ __forceinline__ void bwd_rows(BwdBars* bars, float* row_buf, const fl
                                          const float* __restrict__ Delta, int T, const WorkList& wl, int tid64) {
     volatile int* abort_flag = &bars->abort_flag;
     int g = 0;
-    for (int p = 0; p < wl.passes(); ++p) {
+    for (WorkCursor cur; !wl.done(cur); wl.advance(cur)) {
         int kt, bh, i0, n_it;
-        if (!wl.get(p, &kt, &bh, &i0, &n_it)) continue;
+        if (!wl.get(cur, &kt, &bh, &i0, &n_it)) continue;
         const size_t row_base = static_cast<size_t>(bh) * T;
         for (int it = 0; it < n_it; ++it, ++g) {
             const int b = g & 1;
@@ -474,9 +487,9 @@ __device__ __forceinline__ void bwd_compute(uint8_t* smem, BwdBars* bars, uint32
     bool ok = true;
     int w = 0, g = 0;
 
-    for (int p = 0; p < wl.passes() && ok; ++p) {
+    for (WorkCursor cur; !wl.done(cur) && ok; wl.advance(cur)) {
         int kt, bh, i0, n_it;
-        if (!wl.get(p, &kt, &bh, &i0, &n_it)) continue;
+        if (!wl.get(cur, &kt, &bh, &i0, &n_it)) continue;
         const int key = kt * kBlockK + r;
         const bool key_valid = key < T;
         const bool tile_keys_valid = (kt * kBlockK + kBlockK) <= T;
@@ -561,14 +574,14 @@ __device__ __forceinline__ void bwd_compute(uint8_t* smem, BwdBars* bars, uint32
                     dd[2 * y + 1] = pack_bf16x2(d2, d3);
                 }
                 if (x + 16 < kQPT) tmem_ld_x16(t_dp + x + 16, dv);  // all of dv has been consumed above
-                tmem_st_x8(t_dp + x / 2, dd);
-                if (!wl.no_dq) {  // dS^T row r: two 16-byte chunks of one 128-byte swizzled row
+                if (!Cfg::kdKFromSmem) tmem_st_x8(t_dp + x / 2, dd);
+                if (Cfg::kdKFromSmem || !wl.no_dq()) {  // dS^T row r: two 16-byte chunks of one 128-byte swizzled row
                     const int ch = ch0 + x / 8;
                     *reinterpret_cast<uint4*>(sdS_row + (((ch + 0) ^ (r & 7)) << 4)) = make_uint4(dd[0], dd[1], dd[2], dd[3]);
                     *reinterpret_cast<uint4*>(sdS_row + (((ch + 1) ^ (r & 7)) << 4)) = make_uint4(dd[4], dd[5], dd[6], dd[7]);
                 }
             }
-            tmem_wait_st();
+            if (!Cfg::kdKFromSmem) tmem_wait_st();
             fence_proxy_async_smem();
             tc_fence_before();
             __syncwarp();
@@ -586,7 +599,7 @@ __device__ __forceinline__ void bwd_compute(uint8_t* smem, BwdBars* bars, uint32
             ok = mbar_wait(&bars->dkv_full, w & 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
-            const long long hb = bh % wl.H, bb = bh / wl.H;
+            const long long hb = bh % wl.H(), bb = bh / wl.H();
             uint4* dv_row = reinterpret_cast<uint4*>(dV + bb * sdv.b + hb * sdv.h + key * sdv.t + half * kColsPerThread);
             uint4* dk_row = reinterpret_cast<uint4*>(dK + bb * sdk.b + hb * sdk.h + key * sdk.t + half * kColsPerThread);
 #pragma unroll
@@ -646,9 +659,9 @@ __device__ __forceinline__ void bwd_dq_tma(uint8_t* smem, BwdBars* bars, uint32_
                     tma_reduce_add_3d(tmAcc, stage, 0, row, bh);
                     tma_reduce_add_3d(tmAcc, stage + kHalfTileBytes, 32, row, bh);
                 } else {
-                    const int hh = kStrided ? bh % wl.H : 0, bb = kStrided ? bh / wl.H : 0;
-                    tma_store_tile<kStrided>(tmdV, stage, (wl.orders >> 20) & 15, 0, row, hh, bb, bh);
-                    tma_store_tile<kStrided>(tmdK, stage + kHalfTileBytes, (wl.orders >> 16) & 15, 0, row, hh, bb, bh);
+                    const int hh = kStrided ? bh % wl.H() : 0, bb = kStrided ? bh / wl.H() : 0;
+                    tma_store_tile<kStrided>(tmdV, stage, (wl.orders() >> 20) & 15, 0, row, hh, bb, bh);
+                    tma_store_tile<kStrided>(tmdK, stage + kHalfTileBytes, (wl.orders() >> 16) & 15, 0, row, hh, bb, bh);
                 }
                 bulk_commit_group();
             }
@@ -672,10 +685,10 @@ __device__ __forceinline__ void bwd_dq_tma(uint8_t* smem, BwdBars* bars, uint32_
         return mbar_wait(&bars->stage_free, (u - 1) & 1, abort_flag);
     };
 
-    for (int p = 0; p < wl.passes() && ok; ++p) {
+    for (WorkCursor cur; !wl.done(cur) && ok; wl.advance(cur)) {
         int kt, bh, i0, n_it;
-        if (!wl.get(p, &kt, &bh, &i0, &n_it)) continue;
-        for (int it = 0; it < n_it && !wl.no_dq; ++it, ++g) {
+        if (!wl.get(cur, &kt, &bh, &i0, &n_it)) continue;
+        for (int it = 0; it < n_it && !wl.no_dq(); ++it, ++g) {
             ok = mbar_wait(&bars->dq_full, g & 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
@@ -742,10 +755,11 @@ __device__ __forceinline__ void bwd_dq_tma(uint8_t* smem, BwdBars* bars, uint32_
 }
 
 // dQ warps at D=128.  One thread per query row; the partial dQ tile is 128 fp32 columns, i.e. four
-// boxes of the accumulator's tensor map.  They leave TMEM two at a time (64 registers), go through the
-// two halves of the staging buffer and out with one TMA reduce-add each; the dQ columns are released
-// as soon as the second pair has been loaded, and a half of the buffer is refilled once the copy
-// engine has read the box before last.
+// boxes of the accumulator's tensor map, and the staging buffer holds two.  The dQ columns are the dP^T
+// columns of the next tile, so how soon they are handed back sets the period of a tile: the first 64
+// columns go straight into the two halves of the staging buffer, the other 64 are loaded into the same
+// registers, and the columns are released before any copy is issued.  Then boxes 0 and 1 leave with one
+// TMA reduce-add each, and boxes 2 and 3 follow through the same halves once the copy engine has read them.
 __device__ __forceinline__ void bwd_dq_tma_wide(uint8_t* smem, BwdBars* bars, uint32_t tmem_base,
                                                 const CUtensorMap* tmAcc, const WorkList& wl, int qwarp, int lane) {
     constexpr int D = 128;
@@ -756,63 +770,75 @@ __device__ __forceinline__ void bwd_dq_tma_wide(uint8_t* smem, BwdBars* bars, ui
     const bool leader = (qwarp == 0 && lane == 0);
     const uint32_t t_dq = tmem_addr(tmem_base, lane_base, Cfg::kColdQ);
     uint8_t* stage = smem + Cfg::kOffStage;
+    uint8_t* row_ptr = stage + r * 128;
     const int sw = r & 7;
     bool ok = true;
-    int g = 0, u = 0;  // query tiles, boxes sent so far
+    int g = 0, nf = 0, nr = 0;  // query tiles; uses of stage_full and of stage_free so far
 
-    // Sends 32 accumulator columns (one box) of this thread's row through half (u & 1) of the buffer.
-    auto send_box = [&](const uint32_t* a, int col, int row, int bh) -> bool {
-        if (u >= 2) {  // the box before last used this half: the copy engine must have read it
-            if (leader) {
-                bulk_wait_group_read<1>();
-                mbar_arrive(&bars->stage_free);
-            }
-            __syncwarp();
-            if (!mbar_wait(&bars->stage_free, (u - 2) & 1, abort_flag)) return false;
-        }
-        uint8_t* box = stage + (u & 1) * kHalfTileBytes;
-        uint8_t* row_ptr = box + r * 128;
+    // 64 columns of this thread's row into the two halves of the staging buffer (one box each).
+    auto fill = [&](const uint32_t* a) {
 #pragma unroll
-        for (int ch = 0; ch < 8; ++ch)
-            *reinterpret_cast<uint4*>(row_ptr + ((ch ^ sw) << 4)) =
-                make_uint4(a[ch * 4], a[ch * 4 + 1], a[ch * 4 + 2], a[ch * 4 + 3]);
+        for (int hb = 0; hb < 2; ++hb)
+#pragma unroll
+            for (int ch = 0; ch < 8; ++ch)
+                *reinterpret_cast<uint4*>(row_ptr + hb * kHalfTileBytes + ((ch ^ sw) << 4)) =
+                    make_uint4(a[32 * hb + ch * 4], a[32 * hb + ch * 4 + 1], a[32 * hb + ch * 4 + 2], a[32 * hb + ch * 4 + 3]);
+    };
+    // Hands the two filled boxes to the leader, who adds them into the accumulator at columns col, col + 32.
+    auto send = [&](int col, int row, int bh) -> bool {
         fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) mbar_arrive(&bars->stage_full);
         bool leader_ok = true;
         if (leader) {
-            leader_ok = mbar_wait(&bars->stage_full, u & 1, abort_flag);
+            leader_ok = mbar_wait(&bars->stage_full, nf & 1, abort_flag);
             if (leader_ok) {
-                tma_reduce_add_3d(tmAcc, box, col, row, bh);
+                tma_reduce_add_3d(tmAcc, stage, col, row, bh);
+                tma_reduce_add_3d(tmAcc, stage + kHalfTileBytes, col + 32, row, bh);
                 bulk_commit_group();
             }
         }
-        ++u;
+        ++nf;
         return __all_sync(0xffffffffu, leader_ok);
     };
+    // Before the staging buffer is refilled the copy engine must have read what was sent from it.
+    auto reusable = [&]() -> bool {
+        if (leader) {
+            bulk_wait_group_read<0>();
+            mbar_arrive(&bars->stage_free);
+        }
+        __syncwarp();
+        const bool fine = mbar_wait(&bars->stage_free, nr & 1, abort_flag);
+        ++nr;
+        return __all_sync(0xffffffffu, fine);  // also brings the warp together before its next TMEM instruction
+    };
 
-    for (int p = 0; p < wl.passes() && ok && !wl.no_dq; ++p) {
+    for (WorkCursor cur; !wl.done(cur) && ok && !wl.no_dq(); wl.advance(cur)) {
         int kt, bh, i0, n_it;
-        if (!wl.get(p, &kt, &bh, &i0, &n_it)) continue;
+        if (!wl.get(cur, &kt, &bh, &i0, &n_it)) continue;
         for (int it = 0; it < n_it && ok; ++it, ++g) {
             ok = mbar_wait(&bars->dq_full, g & 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
             const int row = (i0 + it) * kBlockQ;
-#pragma unroll
-            for (int half = 0; half < 2 && ok; ++half) {
-                uint32_t a[64];
-                tmem_ld_x32(t_dq + 64 * half, a);
-                tmem_ld_x32(t_dq + 64 * half + 32, a + 32);
-                tmem_wait_ld();
-                if (half == 1) {  // the whole tile has left TMEM
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&bars->dq_free);
-                }
-                ok = send_box(a, 64 * half, row, bh);
-                if (ok) ok = send_box(a + 32, 64 * half + 32, row, bh);
-            }
+            uint32_t a[64];
+            tmem_ld_x32(t_dq, a);
+            tmem_ld_x32(t_dq + 32, a + 32);
+            if (g > 0) ok = reusable();  // the second pair of boxes of the previous tile, sent most of a tile ago
+            tmem_wait_ld();
+            if (!ok) break;
+            fill(a);
+            tmem_ld_x32(t_dq + 64, a);
+            tmem_ld_x32(t_dq + 96, a + 32);
+            tmem_wait_ld();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bars->dq_free);  // the whole tile has left TMEM
+            ok = send(0, row, bh);
+            if (ok) ok = reusable();
+            if (!ok) break;
+            fill(a);
+            ok = send(64, row, bh);
         }
     }
     // Also when giving up: nothing of this thread may stay in flight, and the accumulator must be
@@ -827,8 +853,8 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 const __grid_constant__ CUtensorMap tmAcc, const __grid_constant__ CUtensorMap tmdK,
                 const __grid_constant__ CUtensorMap tmdV, const float* __restrict__ LSE,
                 const float* __restrict__ Delta, __nv_bfloat16* __restrict__ dK,
-                __nv_bfloat16* __restrict__ dV, const TensorStrides sdk, const TensorStrides sdv, int T, int BH,
-                int H, uint32_t orders, int no_dq, int n_tiles, float scale, int* __restrict__ dev_status) {
+                __nv_bfloat16* __restrict__ dV, const TensorStrides sdk, const TensorStrides sdv, int T,
+                const __grid_constant__ WorkArgs wa, float scale, int* __restrict__ dev_status) {
     using Cfg = BwdCfg<D>;
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -841,8 +867,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     }
     BwdBars* bars = reinterpret_cast<BwdBars*>(smem + Cfg::kOffBar);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const WorkList wl{n_tiles * BH, static_cast<int>(gridDim.x), static_cast<int>(blockIdx.x), BH, n_tiles, H, orders,
-                      no_dq != 0, kCausal};
+    const WorkList wl{wa, kCausal};
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < 2; ++s) {
@@ -891,14 +916,14 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     griddep_launch_dependents();
     if (warp == 0 && lane == 0) {  // the first item's K, V and first Q, dO tiles on their way into L2 meanwhile
         int kt, bh, i0, n_it;
-        if (wl.get(0, &kt, &bh, &i0, &n_it)) {
-            const int head = kStrided ? bh % wl.H : 0, batch = kStrided ? bh / wl.H : 0;
+        if (wl.get(WorkCursor{}, &kt, &bh, &i0, &n_it)) {
+            const int head = kStrided ? bh % wl.H() : 0, batch = kStrided ? bh / wl.H() : 0;
 #pragma unroll
             for (int h = 0; h < Cfg::kHalves; ++h) {
-                tma_prefetch_tile<kStrided>(&tmK, (wl.orders >> 4) & 15, h * kBoxCols, kt * kBlockK, head, batch, bh);
-                tma_prefetch_tile<kStrided>(&tmQ, wl.orders & 15, h * kBoxCols, i0 * kBlockQ, head, batch, bh);
-                tma_prefetch_tile<kStrided>(&tmV, (wl.orders >> 8) & 15, h * kBoxCols, kt * kBlockK, head, batch, bh);
-                tma_prefetch_tile<kStrided>(&tmdO, (wl.orders >> 12) & 15, h * kBoxCols, i0 * kBlockQ, head, batch, bh);
+                tma_prefetch_tile<kStrided>(&tmK, (wl.orders() >> 4) & 15, h * kBoxCols, kt * kBlockK, head, batch, bh);
+                tma_prefetch_tile<kStrided>(&tmQ, wl.orders() & 15, h * kBoxCols, i0 * kBlockQ, head, batch, bh);
+                tma_prefetch_tile<kStrided>(&tmV, (wl.orders() >> 8) & 15, h * kBoxCols, kt * kBlockK, head, batch, bh);
+                tma_prefetch_tile<kStrided>(&tmdO, (wl.orders() >> 12) & 15, h * kBoxCols, i0 * kBlockQ, head, batch, bh);
             }
         }
     }
@@ -931,17 +956,19 @@ cudaError_t launch_one(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUt
                        const CUtensorMap& tmdV, bool strided, uint32_t orders, bool no_dq, const float* LSE,
                        const float* Delta, __nv_bfloat16* dK, __nv_bfloat16* dV, const TensorStrides& sdk,
                        const TensorStrides& sdv, const AttnShape& s, int num_sms, int* dev_status, cudaStream_t stream) {
-    const int n_tiles = (s.T + kBlockK - 1) / kBlockK;
+    static_assert(kBlockK == 128 && kBlockQ == 128, "the work plan counts 128-row tiles");
     const int BH = s.B * s.H;
-    const long long n_items = static_cast<long long>(n_tiles) * BH;
-    const dim3 grid(static_cast<unsigned>(n_items < num_sms ? n_items : num_sms));  // one persistent CTA per SM
+    int n_tiles = 0, n_ctas = 0;
+    const WorkPlan plan = bwd_work_plan(BH, s.T, D, kCausal, num_sms, &n_tiles, &n_ctas);
+    const dim3 grid(static_cast<unsigned>(n_ctas));  // one persistent CTA per SM
+    const WorkArgs wa{BH, n_tiles, s.H, orders, no_dq ? 1 : 0, plan};
     if (strided)
         return launch_overlapped(attn_bwd_kernel<D, kCausal, true>, grid, dim3(BwdCfg<D>::kThreads), BwdCfg<D>::kSmemBytes,
-                                 stream, tmQ, tmK, tmV, tmdO, tmAcc, tmdK, tmdV, LSE, Delta, dK, dV, sdk, sdv, s.T, BH, s.H,
-                                 orders, no_dq ? 1 : 0, n_tiles, s.scale, dev_status);
+                                 stream, tmQ, tmK, tmV, tmdO, tmAcc, tmdK, tmdV, LSE, Delta, dK, dV, sdk, sdv, s.T, wa,
+                                 s.scale, dev_status);
     return launch_overlapped(attn_bwd_kernel<D, kCausal, false>, grid, dim3(BwdCfg<D>::kThreads), BwdCfg<D>::kSmemBytes, stream,
-                             tmQ, tmK, tmV, tmdO, tmAcc, tmdK, tmdV, LSE, Delta, dK, dV, sdk, sdv, s.T, BH, s.H, orders,
-                             no_dq ? 1 : 0, n_tiles, s.scale, dev_status);
+                             tmQ, tmK, tmV, tmdO, tmAcc, tmdK, tmdV, LSE, Delta, dK, dV, sdk, sdv, s.T, wa, s.scale,
+                             dev_status);
 }
 
 template <int D, bool kCausal, bool kStrided>

@@ -77,6 +77,8 @@ def load():
     lib.nova_attn_static_scratch_bytes.restype = sz
     lib.nova_attn_test_configure_waits.argtypes = [ctypes.c_longlong, i]
     lib.nova_attn_test_configure_waits.restype = i
+    lib.nova_attn_bwd_work_list.argtypes = [i, ctypes.c_longlong, i, i, i, i, ctypes.c_void_p, i, ctypes.c_void_p]
+    lib.nova_attn_bwd_work_list.restype = i
     _lib = lib
     return lib
 
@@ -217,6 +219,21 @@ def nova_attn_test_configure_waits(limit_cycles: int = 0, inject: int = 0) -> No
     rc = load().nova_attn_test_configure_waits(int(limit_cycles), int(inject))
     if rc != OK:
         raise NovaAttnError(rc, "nova_attn_test_configure_waits")
+
+
+def nova_attn_bwd_work_list(BH: int, T: int, D: int, causal: bool, n_ctas: int, cta: int):
+    """Host-side view of the backward kernel's work distribution: ([(key tile, head), ...] of CTA `cta` in
+    processing order, (heads per chunk, chunks, passes per full chunk, passes of the last chunk)).  No GPU."""
+    lib = load()
+    plan = (ctypes.c_int * 4)()
+    n = lib.nova_attn_bwd_work_list(int(BH), int(T), int(D), int(bool(causal)), int(n_ctas), int(cta), None, 0, plan)
+    if n < 0:
+        raise NovaAttnError(n, "nova_attn_bwd_work_list")
+    buf = (ctypes.c_int * (2 * max(n, 1)))()
+    m = lib.nova_attn_bwd_work_list(int(BH), int(T), int(D), int(bool(causal)), int(n_ctas), int(cta), buf, n, plan)
+    if m != n:
+        raise NovaAttnError(ERR_SHAPE if m >= 0 else m, "nova_attn_bwd_work_list")
+    return [(buf[2 * k], buf[2 * k + 1]) for k in range(n)], tuple(plan)
 
 
 def nova_attn_poll_device_status(stream=None) -> int:
