@@ -39,6 +39,8 @@
 //
 // Warp-wide .sync.aligned instructions (TMEM loads/stores) need the whole warp together: wherever
 // one lane does extra work (the dQ leader), the warp is rejoined with a vote before the next one.
+#include <type_traits>
+
 #include "kernels.h"
 #include "ptx.cuh"
 #include "work_plan.h"
@@ -758,8 +760,11 @@ __device__ __forceinline__ void bwd_dq_tma(uint8_t* smem, BwdBars* bars, uint32_
 // boxes of the accumulator's tensor map, and the staging buffer holds two.  The dQ columns are the dP^T
 // columns of the next tile, so how soon they are handed back sets the period of a tile: the first 64
 // columns go straight into the two halves of the staging buffer, the other 64 are loaded into the same
-// registers, and the columns are released before any copy is issued.  Then boxes 0 and 1 leave with one
-// TMA reduce-add each, and boxes 2 and 3 follow through the same halves once the copy engine has read them.
+// registers, and the columns are released before any copy is issued.  A reduction runs at about 25 bytes
+// per clock and SM however it is issued (TMA or red.global, measured), 2600 clocks for the 64 KB of a tile
+// against 2600 clocks of tensor work, so the copy engine must never idle: every box is a bulk group of its
+// own, boxes 0 and 1 are issued together, box 2 goes into the first half as soon as box 0 has been read
+// (box 1 still being read), box 3 into the second half once box 1 has been.
 __device__ __forceinline__ void bwd_dq_tma_wide(uint8_t* smem, BwdBars* bars, uint32_t tmem_base,
                                                 const CUtensorMap* tmAcc, const WorkList& wl, int qwarp, int lane) {
     constexpr int D = 128;
@@ -775,17 +780,16 @@ __device__ __forceinline__ void bwd_dq_tma_wide(uint8_t* smem, BwdBars* bars, ui
     bool ok = true;
     int g = 0, nf = 0, nr = 0;  // query tiles; uses of stage_full and of stage_free so far
 
-    // 64 columns of this thread's row into the two halves of the staging buffer (one box each).
-    auto fill = [&](const uint32_t* a) {
+    // 32 columns of this thread's row into half hb of the staging buffer (one box).
+    auto fill = [&](const uint32_t* a, int hb) {
 #pragma unroll
-        for (int hb = 0; hb < 2; ++hb)
-#pragma unroll
-            for (int ch = 0; ch < 8; ++ch)
-                *reinterpret_cast<uint4*>(row_ptr + hb * kHalfTileBytes + ((ch ^ sw) << 4)) =
-                    make_uint4(a[32 * hb + ch * 4], a[32 * hb + ch * 4 + 1], a[32 * hb + ch * 4 + 2], a[32 * hb + ch * 4 + 3]);
+        for (int ch = 0; ch < 8; ++ch)
+            *reinterpret_cast<uint4*>(row_ptr + hb * kHalfTileBytes + ((ch ^ sw) << 4)) =
+                make_uint4(a[ch * 4], a[ch * 4 + 1], a[ch * 4 + 2], a[ch * 4 + 3]);
     };
-    // Hands the two filled boxes to the leader, who adds them into the accumulator at columns col, col + 32.
-    auto send = [&](int col, int row, int bh) -> bool {
+    // Hands filled boxes to the leader, who adds them into the accumulator: half `first` at column `col`,
+    // and with n = 2 the other half at col + 32; one bulk group per box.
+    auto send = [&](int first, int n, int col, int row, int bh) -> bool {
         fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) mbar_arrive(&bars->stage_full);
@@ -793,18 +797,20 @@ __device__ __forceinline__ void bwd_dq_tma_wide(uint8_t* smem, BwdBars* bars, ui
         if (leader) {
             leader_ok = mbar_wait(&bars->stage_full, nf & 1, abort_flag);
             if (leader_ok) {
-                tma_reduce_add_3d(tmAcc, stage, col, row, bh);
-                tma_reduce_add_3d(tmAcc, stage + kHalfTileBytes, col + 32, row, bh);
-                bulk_commit_group();
+                for (int k = 0; k < n; ++k) {
+                    tma_reduce_add_3d(tmAcc, stage + (first + k) * kHalfTileBytes, col + 32 * k, row, bh);
+                    bulk_commit_group();
+                }
             }
         }
         ++nf;
         return __all_sync(0xffffffffu, leader_ok);
     };
-    // Before the staging buffer is refilled the copy engine must have read what was sent from it.
-    auto reusable = [&]() -> bool {
+    // Before a half of the staging buffer is refilled the copy engine must have read what was sent from it:
+    // all groups (kPending = 0) or all but the latest one (kPending = 1).
+    auto reusable = [&](auto pending) -> bool {
         if (leader) {
-            bulk_wait_group_read<0>();
+            bulk_wait_group_read<decltype(pending)::value>();
             mbar_arrive(&bars->stage_free);
         }
         __syncwarp();
@@ -824,21 +830,26 @@ __device__ __forceinline__ void bwd_dq_tma_wide(uint8_t* smem, BwdBars* bars, ui
             uint32_t a[64];
             tmem_ld_x32(t_dq, a);
             tmem_ld_x32(t_dq + 32, a + 32);
-            if (g > 0) ok = reusable();  // the second pair of boxes of the previous tile, sent most of a tile ago
+            if (g > 0) ok = reusable(std::integral_constant<int, 0>{});  // boxes 2, 3 of the previous tile
             tmem_wait_ld();
             if (!ok) break;
-            fill(a);
+            fill(a, 0);
+            fill(a + 32, 1);
             tmem_ld_x32(t_dq + 64, a);
             tmem_ld_x32(t_dq + 96, a + 32);
             tmem_wait_ld();
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&bars->dq_free);  // the whole tile has left TMEM
-            ok = send(0, row, bh);
-            if (ok) ok = reusable();
+            ok = send(0, 2, 0, row, bh);
+            if (ok) ok = reusable(std::integral_constant<int, 1>{});  // box 0 read, box 1 may still be in flight
             if (!ok) break;
-            fill(a);
-            ok = send(64, row, bh);
+            fill(a, 0);
+            ok = send(0, 1, 64, row, bh);
+            if (ok) ok = reusable(std::integral_constant<int, 1>{});  // box 1 read
+            if (!ok) break;
+            fill(a + 32, 1);
+            ok = send(1, 1, 96, row, bh);
         }
     }
     // Also when giving up: nothing of this thread may stay in flight, and the accumulator must be
