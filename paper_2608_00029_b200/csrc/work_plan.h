@@ -2,6 +2,7 @@
 // Shared by the kernel (device) and by the launch code and the tests (host).
 #pragma once
 #include <cstdint>
+#include <mutex>
 
 namespace nova {
 
@@ -68,8 +69,36 @@ struct WorkList {
     }
 };
 
-// Heads per chunk for a working set of about `budget` bytes, chosen among the nearby sizes for the least
-// idle time in the padded last pass of a chunk.
+inline WorkPlan work_plan_for_chunk(int BH, int n_tiles, int n_ctas, int chunk) {
+    WorkPlan wp;
+    wp.chunk = chunk;
+    wp.n_chunks = (BH + chunk - 1) / chunk;
+    wp.passes_per_chunk = static_cast<int>((static_cast<long long>(chunk) * n_tiles + n_ctas - 1) / n_ctas);
+    const int last = BH - (wp.n_chunks - 1) * chunk;
+    wp.passes_last = static_cast<int>((static_cast<long long>(last) * n_tiles + n_ctas - 1) / n_ctas);
+    return wp;
+}
+
+// Largest load of a CTA over the mean load (in tiles) when the items are dealt out by `wp`.
+inline double work_plan_imbalance(int BH, int n_tiles, bool causal, int n_ctas, const WorkPlan& wp) {
+    const WorkArgs wa{BH, n_tiles, 1, 0u, 0, wp};
+    const WorkList wl{wa, causal};
+    long long total = 0, worst = 0;
+    for (int cta = 0; cta < n_ctas; ++cta) {
+        long long load = 0;
+        for (WorkCursor cur; !wl.done(cur); wl.advance(cur)) {
+            int kt, bh, i0, n_it;
+            if (wl.get_for(cur, n_ctas, cta, &kt, &bh, &i0, &n_it)) load += n_it;
+        }
+        total += load;
+        if (load > worst) worst = load;
+    }
+    return total > 0 ? static_cast<double>(worst) * n_ctas / static_cast<double>(total) : 1.0;
+}
+
+// Heads per chunk for a working set of about `budget` bytes and at least `min_passes` passes per chunk:
+// among up to 32 sizes around that, the one whose dealing leaves the CTAs' loads most even (the loads are
+// counted exactly, by walking every CTA's list).
 inline WorkPlan make_work_plan(int BH, int n_tiles, long long T, int D, bool causal, int n_ctas, long long budget,
                                int min_passes) {
     const long long per_head = T * D * 12;  // fp32 accumulator + Q, K, V, dO
@@ -77,31 +106,25 @@ inline WorkPlan make_work_plan(int BH, int n_tiles, long long T, int D, bool cau
     const long long c_min = (static_cast<long long>(min_passes) * n_ctas + n_tiles - 1) / n_tiles;  // heads for min_passes passes
     if (cb < c_min) cb = c_min;
     if (cb < 1) cb = 1;
-    int best = BH;
-    if (cb * 3 / 2 < BH) {
-        const int n_chunks = static_cast<int>((BH + cb - 1) / cb);
-        const int even = (BH + n_chunks - 1) / n_chunks;
-        double best_cost = 1e30;
-        int lo = even / 2 > 1 ? even / 2 : 1;
-        if (lo < c_min) lo = static_cast<int>(c_min < even ? c_min : even);
-        const int hi = even + even / 4;
-        for (int c = hi; c >= lo; --c) {
-            const long long items = static_cast<long long>(c) * n_tiles;
-            const long long passes = (items + n_ctas - 1) / n_ctas;
-            const double idle = static_cast<double>(passes * n_ctas - items) * (causal ? 1.0 : n_tiles);
-            const double work = static_cast<double>(items) * (causal ? (n_tiles + 1) * 0.5 : n_tiles);
-            // a small penalty on chunks far from the budget on either side
-            const double cost = idle / work + 0.02 * (c > even ? static_cast<double>(c - even) / even : static_cast<double>(even - c) / even);
-            if (cost < best_cost) { best_cost = cost; best = c; }
+    if (cb * 3 / 2 >= BH) return work_plan_for_chunk(BH, n_tiles, n_ctas, BH);  // everything fits: one list
+    const int n_chunks = static_cast<int>((BH + cb - 1) / cb);
+    const int even = (BH + n_chunks - 1) / n_chunks;
+    int lo = even - even / 3 > 1 ? even - even / 3 : 1;
+    if (lo < c_min) lo = static_cast<int>(c_min < even ? c_min : even);
+    const int hi = even + even / 4;
+    const int step = (hi - lo) / 32 + 1;
+    int best = even;
+    double best_cost = 1e30;
+    for (int c = hi; c >= lo; c -= step) {
+        const double imbalance = work_plan_imbalance(BH, n_tiles, causal, n_ctas, work_plan_for_chunk(BH, n_tiles, n_ctas, c));
+        // a small penalty on chunks far from the budget on either side
+        const double cost = imbalance + 0.02 * (c > even ? c - even : even - c) / even;
+        if (cost < best_cost) {
+            best_cost = cost;
+            best = c;
         }
     }
-    WorkPlan wp;
-    wp.chunk = best;
-    wp.n_chunks = (BH + best - 1) / best;
-    wp.passes_per_chunk = static_cast<int>((static_cast<long long>(best) * n_tiles + n_ctas - 1) / n_ctas);
-    const int last = BH - (wp.n_chunks - 1) * best;
-    wp.passes_last = static_cast<int>((static_cast<long long>(last) * n_tiles + n_ctas - 1) / n_ctas);
-    return wp;
+    return work_plan_for_chunk(BH, n_tiles, n_ctas, best);
 }
 
 // The plan the backward launch uses for a problem on a device of `num_sms` SMs: one persistent CTA per SM
@@ -114,7 +137,24 @@ inline WorkPlan bwd_work_plan(int BH, long long T, int D, bool causal, int num_s
     const int grid = static_cast<int>(n_items < num_sms ? n_items : num_sms);
     *n_tiles_out = n_tiles;
     *grid_out = grid;
-    return make_work_plan(BH, n_tiles, T, D, causal, grid, 48ll << 20, 2);
+    // The plan is a pure function of the shape; choosing it walks every item, so the last few are kept.
+    struct Entry {
+        int BH, D, causal, num_sms;
+        long long T;
+        WorkPlan plan;
+        bool valid;
+    };
+    constexpr int kEntries = 16;
+    static Entry cache[kEntries] = {};
+    static int next = 0;
+    static std::mutex mutex;
+    std::lock_guard<std::mutex> lock(mutex);
+    for (const Entry& e : cache)
+        if (e.valid && e.BH == BH && e.T == T && e.D == D && e.causal == (causal ? 1 : 0) && e.num_sms == num_sms) return e.plan;
+    const WorkPlan plan = make_work_plan(BH, n_tiles, T, D, causal, grid, 48ll << 20, 2);
+    cache[next] = Entry{BH, D, causal ? 1 : 0, num_sms, T, plan, true};
+    next = (next + 1) % kEntries;
+    return plan;
 }
 
 }  // namespace nova
