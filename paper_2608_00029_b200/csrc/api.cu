@@ -511,15 +511,16 @@ int nova_lmhead_fwd(const void* X, const void* W, const int* targets, void* logi
     if (int rc = device_state(&st)) return rc;
     int rows_x = 0, rows_w = 0;
     const int box_k = lmhead_boxes(&rows_x, &rows_w);
-    CUtensorMap tmX, tmW, tmL;
+    CUtensorMap tmX, tmW, tmWh, tmL;
     if (int rc = encode_matrix_map(X, M, K, rows_x, box_k, &tmX)) return rc;
     if (int rc = encode_matrix_map(W, N, K, rows_w, box_k, &tmW)) return rc;
+    if (int rc = encode_matrix_map(W, N, K, rows_w / 2, box_k, &tmWh)) return rc;  // half a W tile per CTA of a pair
     if (logits) {
         if (int rc = encode_matrix_map(logits, M, N, 32, 64, &tmL)) return rc;
     } else {
         tmL = tmX;  // never used
     }
-    const cudaError_t e = launch_lmhead(tmX, tmW, tmL, logits != nullptr, targets, lse, loss, M, N, K, workspace,
+    const cudaError_t e = launch_lmhead(tmX, tmW, tmWh, tmL, logits != nullptr, targets, lse, loss, M, N, K, workspace,
                                         st->num_sms, st->dev_status, static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? NOVA_ATTN_OK : fail_cuda(e);
 }

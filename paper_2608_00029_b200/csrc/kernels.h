@@ -98,9 +98,9 @@ cudaError_t configure_attn_bwd();
 // Loss head (lmhead.cu): `tmX` is the 2-D map of X [K, M] with box [64, 128], `tmW` that of W [K, N] with box
 // [64, 256], `tmL` that of the logits [N, M] with box [64, 32] (any valid map if `store_logits` is false), all
 // bf16 with 128-byte swizzle.  Enqueues the fused contraction + statistics kernel and the merge.
-cudaError_t launch_lmhead(const CUtensorMap& tmX, const CUtensorMap& tmW, const CUtensorMap& tmL, bool store_logits,
-                          const int* targets, float* lse, float* loss, int M, int N, int K, void* workspace, int num_sms,
-                          int* dev_status, cudaStream_t stream);
+cudaError_t launch_lmhead(const CUtensorMap& tmX, const CUtensorMap& tmW, const CUtensorMap& tmWh, const CUtensorMap& tmL,
+                          bool store_logits, const int* targets, float* lse, float* loss, int M, int N, int K,
+                          void* workspace, int num_sms, int* dev_status, cudaStream_t stream);
 cudaError_t configure_lmhead();
 size_t lmhead_workspace_bytes(int M, int N);
 // Rows of the X and W boxes; returns the box width in k elements.
