@@ -470,6 +470,15 @@ def run_lmhead(args):
     if rank == 0:
         peak = peaks["bf16_tflops"]
         ach = cfg.flops / (ms * 1e-3) / 1e12
+        # DRAM bytes of one launch of the main kernel from the committed ncu summary of this very workload
+        traffic, traffic_source = None, None
+        traffic_rel = os.path.join("profiles", f"lmhead_pair_kernel_{cfg.name}.md")
+        if os.path.exists(os.path.join(ROOT, traffic_rel)):
+            with open(os.path.join(ROOT, traffic_rel)) as f:
+                for ln in f:
+                    if ln.startswith("traffic_bytes_per_launch:"):
+                        traffic = int(ln.split(":")[1])
+                        traffic_source = f"{traffic_rel} (committed ncu summary, not measured in this run)"
         line = {
             "metric": "lm_head_fused_tflops", "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
@@ -484,8 +493,9 @@ def run_lmhead(args):
                     "ms_per_step": e2e_ms, "steps": n_e2e},
             "gpu_launches": 2 * args.steps,
             "clocks": sampler.summary(t0, t1),
-            "roofline": {"bound": "tensor", "kernel": "lmhead_kernel (+ lmhead_merge_kernel)", "achieved": ach, "peak": peak,
-                         "unit": UNIT, "frac": ach / peak, "traffic": None, "peak_source": f"{peak_src} bf16_tflops (burst)",
+            "roofline": {"bound": "tensor", "kernel": "lmhead_pair_kernel (+ lmhead_merge_kernel)", "achieved": ach,
+                         "peak": peak, "unit": UNIT, "frac": ach / peak, "traffic": traffic, "traffic_source": traffic_source,
+                         "peak_source": f"{peak_src} bf16_tflops (burst)",
                          "ms_per_launch": ms, "ms_without_logits": ms_nolog,
                          "library_context": {"what": "torch.matmul alone / torch.matmul + logsumexp over the stored logits",
                                              "ms_gemm": ms_lib_gemm, "ms_gemm_plus_reduction": ms_lib_chain}},
