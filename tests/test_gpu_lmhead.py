@@ -100,3 +100,40 @@ def test_full_size_on_sampled_rows():
     assert ((lse - tl) - loss).abs().max() <= 2.0 ** -8 * tl.abs().max() + 1e-3
     mx = lg.max(dim=1).values
     assert bool((lse >= mx - 2.0 ** -7 * mx.abs() - 1e-3).all()) and bool((lse <= mx + np.log(cfg.N) + 1e-2).all())
+
+
+def test_both_kernels_agree_and_cuda_graph_replay():
+    """M <= 128 runs one CTA per tile, larger M one pair of CTAs per 256-row tile: the same rows must come out the
+    same either way (a row's statistics do not depend on its neighbours), also when the calls are captured into
+    a CUDA graph once and replayed (cluster launches inside a graph), and on a side stream."""
+    from paper_2608_00029_b200 import nova_attn as na, nova_lmhead as lm
+    dev = torch.device("cuda:0")
+    cfg = W.LmHeadConfig("both", M=640, N=1536, K=192, seed=9, w_factor=0.2, ignored_every=11)
+    X, Wm, t = W.make_lmhead_inputs(cfg)
+    x, w, tt = X.to(dev), Wm.to(dev), t.to(dev)
+    ws = torch.empty(lm.nova_lmhead_workspace_bytes(cfg.M, cfg.N, cfg.K), dtype=torch.uint8, device=dev)
+    logits = torch.empty((cfg.M, cfg.N), dtype=torch.bfloat16, device=dev)
+    lse, loss = torch.empty(cfg.M, device=dev), torch.empty(cfg.M, device=dev)
+    lm.nova_lmhead_fwd(x, w, tt, logits, lse, loss, ws)
+    na.nova_attn_poll_device_status()
+    # the first 100 rows alone (one tile of rows: the single-CTA kernel)
+    l1, s1, o1 = torch.empty((100, cfg.N), dtype=torch.bfloat16, device=dev), torch.empty(100, device=dev), torch.empty(100, device=dev)
+    lm.nova_lmhead_fwd(x[:100].contiguous(), w, tt[:100].contiguous(), l1, s1, o1)
+    na.nova_attn_poll_device_status()
+    assert torch.equal(l1, logits[:100]) and torch.equal(s1, lse[:100]) and torch.equal(o1, loss[:100])
+    # captured once, replayed three times on a side stream
+    side = torch.cuda.Stream()
+    lse2, loss2, logits2 = torch.zeros_like(lse), torch.zeros_like(loss), torch.zeros_like(logits)
+    with torch.cuda.stream(side):
+        lm.nova_lmhead_fwd(x, w, tt, logits2, lse2, loss2, ws, stream=side)
+    side.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        lm.nova_lmhead_fwd(x, w, tt, logits2, lse2, loss2, ws, stream=torch.cuda.current_stream())
+    for _ in range(3):
+        lse2.zero_(); loss2.zero_(); logits2.zero_()
+        torch.cuda.synchronize()
+        graph.replay()
+        torch.cuda.synchronize()
+        na.nova_attn_poll_device_status()
+        assert torch.equal(lse2, lse) and torch.equal(loss2, loss) and torch.equal(logits2, logits)
