@@ -109,24 +109,6 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
     }
 }
 
-// The same bounded wait for a role that can afford to notice the completion up to `sleep_ns` late (a
-// loader running stages ahead): it sleeps between two tests instead of polling, so that it takes next to no
-// issue slots from the warps that share its scheduler.
-__device__ __forceinline__ bool mbar_wait_relaxed(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
-                                                  long long limit, unsigned sleep_ns) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const long long t0 = clock64();
-    for (;;) {
-        __nanosleep(sleep_ns);
-        if (mbar_try_wait(bar, parity)) return true;
-        if (*abort_flag != 0) return false;
-        if (clock64() - t0 > limit) {
-            *abort_flag = 1;
-            return false;
-        }
-    }
-}
-
 // ------------------------------------------------------------------ dynamic work distribution
 // A persistent CTA that has finished its work item asks the hardware to cancel the launch of a CTA of the same
 // grid that has not started yet and takes over that CTA's index (sm_100 cluster launch control).  The grid is
