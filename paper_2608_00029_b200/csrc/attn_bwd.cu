@@ -111,6 +111,7 @@ struct BwdBars {
     uint64_t stage_full, stage_free;  // dQ warps <-> their leader thread
     uint64_t dkv_full, dkv_free;      // UMMA -> readers: dV/dK of an item complete; readers -> UMMA: read out
     uint64_t drain;
+    uint64_t out_sync;  // the compute warps among themselves, at the end of an item (D=128)
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -445,32 +446,12 @@ __device__ __forceinline__ void bwd_p_phase(uint32_t (&sv)[N], const float4* s_l
     }
 }
 
-// Converts 32 accumulator columns of dV (as is) and dK (times scale) to bf16 and stores them.
-__device__ __forceinline__ void bwd_store_dkv32(const uint32_t (&a)[32], const uint32_t (&bq)[32], float scale,
-                                                uint4* dv_row, uint4* dk_row) {
-#pragma unroll
-    for (int x = 0; x < 32; x += 8) {
-        uint4 v, u;
-        v.x = pack_bf16x2(__uint_as_float(a[x + 0]), __uint_as_float(a[x + 1]));
-        v.y = pack_bf16x2(__uint_as_float(a[x + 2]), __uint_as_float(a[x + 3]));
-        v.z = pack_bf16x2(__uint_as_float(a[x + 4]), __uint_as_float(a[x + 5]));
-        v.w = pack_bf16x2(__uint_as_float(a[x + 6]), __uint_as_float(a[x + 7]));
-        u.x = pack_bf16x2(__uint_as_float(bq[x + 0]) * scale, __uint_as_float(bq[x + 1]) * scale);
-        u.y = pack_bf16x2(__uint_as_float(bq[x + 2]) * scale, __uint_as_float(bq[x + 3]) * scale);
-        u.z = pack_bf16x2(__uint_as_float(bq[x + 4]) * scale, __uint_as_float(bq[x + 5]) * scale);
-        u.w = pack_bf16x2(__uint_as_float(bq[x + 6]) * scale, __uint_as_float(bq[x + 7]) * scale);
-        dv_row[x / 8] = v;
-        dk_row[x / 8] = u;
-    }
-}
-
 // Compute warps.  A thread owns one key row and kQPT consecutive queries of the tile (64: two warpgroups;
 // 32: four), i.e. columns [kQPT*part, kQPT*(part+1)) of S^T and dP^T.
-template <int D, bool kCausal>
-__device__ __forceinline__ void bwd_compute(uint8_t* smem, BwdBars* bars, uint32_t tmem_base,
-                                            __nv_bfloat16* __restrict__ dK, __nv_bfloat16* __restrict__ dV,
-                                            const TensorStrides& sdk, const TensorStrides& sdv, int T, float scale,
-                                            const WorkList& wl, int cwarp, int lane) {
+template <int D, bool kCausal, bool kStrided>
+__device__ __forceinline__ void bwd_compute(uint8_t* smem, BwdBars* bars, uint32_t tmem_base, const CUtensorMap* tmdK,
+                                            const CUtensorMap* tmdV, int T, float scale, const WorkList& wl, int cwarp,
+                                            int lane) {
     using Cfg = BwdCfg<D>;
     constexpr int kQPT = Cfg::kQPT;
     volatile int* abort_flag = &bars->abort_flag;
@@ -488,6 +469,7 @@ __device__ __forceinline__ void bwd_compute(uint8_t* smem, BwdBars* bars, uint32
     const int ch0 = ((part * kQPT) % 64) / 8;  // first 16-byte chunk of this thread's queries in the 128-byte row
     bool ok = true;
     int w = 0, g = 0;
+    int n_sync = 0;  // uses of out_sync so far
 
     for (WorkCursor cur; !wl.done(cur) && ok; wl.advance(cur)) {
         int kt, bh, i0, n_it;
@@ -594,30 +576,73 @@ __device__ __forceinline__ void bwd_compute(uint8_t* smem, BwdBars* bars, uint32
         }
         if (!ok) break;
         if constexpr (!Cfg::kBulkdQ) {
-            // ---- end of the item (D=128): dV and dK of this key row, D/2 columns of each per thread.
+            // ---- end of the item (D=128): dV, then dK (scaled), of this key row, D/2 columns of each per thread,
+            // rounded to bf16 into the dS^T staging buffer (idle now: every product of the item has completed)
+            // as two boxes of [128 keys x 64 columns], and out with two TMA stores each.  (Stores of 16 bytes
+            // per thread straight to global memory, 256 bytes apart, took 5700 clocks per item and held up the
+            // loads of the next item behind them.)
             constexpr int kColsPerThread = D / 2;
             const uint32_t t_dv = tmem_addr(tmem_base, lane_base, Cfg::kColdV + half * kColsPerThread);
             const uint32_t t_dk = tmem_addr(tmem_base, lane_base, Cfg::kColdK + half * kColsPerThread);
             ok = mbar_wait(&bars->dkv_full, w & 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
-            const long long hb = bh % wl.H(), bb = bh / wl.H();
-            uint4* dv_row = reinterpret_cast<uint4*>(dV + bb * sdv.b + hb * sdv.h + key * sdv.t + half * kColsPerThread);
-            uint4* dk_row = reinterpret_cast<uint4*>(dK + bb * sdk.b + hb * sdk.h + key * sdk.t + half * kColsPerThread);
+            const int hh = kStrided ? bh % wl.H() : 0, bb = kStrided ? bh / wl.H() : 0;
+            uint8_t* out_row = smem + Cfg::kOffdS + half * kHalfTileBytes + r * 128;
+            const bool store_leader = (cwarp == 0 && lane == 0);
+            // all compute warps together (bounded, like every wait here)
+            auto all_warps = [&]() -> bool {
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&bars->out_sync);
+                const bool fine = mbar_wait(&bars->out_sync, n_sync & 1, abort_flag);
+                ++n_sync;
+                return fine;
+            };
 #pragma unroll
-            for (int cb = 0; cb < kColsPerThread; cb += 32) {
-                uint32_t a[32], bq[32];
-                tmem_ld_x32(t_dv + cb, a);
-                tmem_ld_x32(t_dk + cb, bq);
+            for (int which = 0; which < 2 && ok; ++which) {
+                uint32_t a[kColsPerThread];
+                const uint32_t t_src = which ? t_dk : t_dv;
+#pragma unroll
+                for (int cb = 0; cb < kColsPerThread; cb += 32) tmem_ld_x32(t_src + cb, a + cb);
                 tmem_wait_ld();
-                if (key_valid) bwd_store_dkv32(a, bq, scale, dv_row + cb / 8, dk_row + cb / 8);
+                if (which == 1) {  // both accumulators have left tensor memory
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&bars->dkv_free);
+                    // the buffer holds dV until the copy engine has read it
+                    if (store_leader) bulk_wait_group_read<0>();
+                    ok = all_warps();
+                    if (!ok) break;
+                }
+                const float f = which ? scale : 1.0f;
+#pragma unroll
+                for (int ch = 0; ch < kColsPerThread / 8; ++ch)
+                    *reinterpret_cast<uint4*>(out_row + ((ch ^ (r & 7)) << 4)) = make_uint4(
+                        pack_bf16x2(__uint_as_float(a[8 * ch + 0]) * f, __uint_as_float(a[8 * ch + 1]) * f),
+                        pack_bf16x2(__uint_as_float(a[8 * ch + 2]) * f, __uint_as_float(a[8 * ch + 3]) * f),
+                        pack_bf16x2(__uint_as_float(a[8 * ch + 4]) * f, __uint_as_float(a[8 * ch + 5]) * f),
+                        pack_bf16x2(__uint_as_float(a[8 * ch + 6]) * f, __uint_as_float(a[8 * ch + 7]) * f));
+                fence_proxy_async_smem();
+                ok = all_warps();
+                if (!ok) break;
+                if (store_leader) {
+                    const CUtensorMap* tm = which ? tmdK : tmdV;
+                    const int order = which ? (wl.orders() >> 16) & 15 : (wl.orders() >> 20) & 15;
+                    tma_store_tile<kStrided>(tm, smem + Cfg::kOffdS, order, 0, kt * kBlockK, hh, bb, bh);
+                    tma_store_tile<kStrided>(tm, smem + Cfg::kOffdS + kHalfTileBytes, order, kBoxCols, kt * kBlockK, hh, bb, bh);
+                    bulk_commit_group();
+                }
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&bars->dkv_free);
+            if (!ok) break;
+            // the next item's dS phase writes this buffer: the copy engine must have read dK
+            if (store_leader) bulk_wait_group_read<0>();
+            ok = all_warps();
+            if (!ok) break;
         }
         ++w;
     }
+    // Also when giving up: the stores of dV and dK must be complete before the kernel ends.
+    if (!Cfg::kBulkdQ && cwarp == 0 && lane == 0) bulk_wait_group<0>();
 }
 
 // dQ warps at D=64.  One thread per row.  Per query tile they move the partial dQ tile from TMEM into
@@ -906,6 +931,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         mbar_init(&bars->dkv_full, 1);
         mbar_init(&bars->dkv_free, Cfg::kBulkdQ ? 4 : Cfg::kComputeWarps);
         mbar_init(&bars->drain, 1);
+        mbar_init(&bars->out_sync, Cfg::kComputeWarps);
         bars->abort_flag = 0;
         fence_mbar_init();
         tma_prefetch_desc(&tmQ);
@@ -947,7 +973,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     } else if (warp < 4) {
         bwd_rows(bars, reinterpret_cast<float*>(smem + Cfg::kOffRow), LSE, Delta, T, wl, (warp - 2) * 32 + lane);
     } else if (warp < 4 + Cfg::kComputeWarps) {
-        bwd_compute<D, kCausal>(smem, bars, tmem_base, dK, dV, sdk, sdv, T, scale, wl, warp - 4, lane);
+        bwd_compute<D, kCausal, kStrided>(smem, bars, tmem_base, &tmdK, &tmdV, T, scale, wl, warp - 4, lane);
     } else {
         if constexpr (Cfg::kBulkdQ)
             bwd_dq_tma<kStrided>(smem, bars, tmem_base, &tmAcc, &tmdK, &tmdV, scale, wl, warp - 4 - Cfg::kComputeWarps, lane);
