@@ -24,7 +24,7 @@
 //                work on the next P
 //   warps 2-3    row loader: -LSE*log2e and -Delta of the query tile into shared memory
 //   warps 4-11   compute: thread = (key row, 64-query half); P phase then dS phase per tile
-//                (at D=128 they also write dV and dK at the end of an item)
+//                (at D=128 they also send dV and dK at the end of an item, through the dS^T staging buffer)
 //   warps 12-15  dQ: one thread per row moves the partial dQ tile from TMEM into the fp32 accumulator
 //                with TMA reduce-add operations through a swizzled staging buffer (a separate kernel
 //                scales and rounds it once); at D=64 they also send dV and dK
