@@ -298,7 +298,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ C
 //              name a barrier of the peer).  One commit signals the `empty` (and `acc_full`) barriers of both.
 //   warps 2-9  epilogue on the CTA's own 128 rows, as above; the peer's warps release an accumulator buffer by
 //              arriving on the leader's barrier
-// No multicast loads: each CTA fetches what it needs itself.
+// Every CTA fetches what it needs itself: no copy is shared between the two.
 constexpr int kPairStages = 6;
 constexpr int kPairWBytes = (kBN / 2) * kBK * 2;
 constexpr int kPairStageBytes = kABytes + kPairWBytes;
@@ -354,7 +354,7 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity
     }
 }
 // 2-D tiled load into this CTA's shared memory whose bytes are counted on a barrier given by its address in
-// the cluster's shared window (the leader's, for both CTAs of a pair).  No multicast.
+// the cluster's shared window (the leader's, for both CTAs of a pair).  The data go to this CTA only.
 __device__ __forceinline__ void tma_load_2d_pair(void* smem_dst, const CUtensorMap* m, uint32_t bar_cluster_addr, int c0,
                                                  int c1) {
     asm volatile(
