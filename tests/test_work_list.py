@@ -73,3 +73,33 @@ def test_bad_arguments():
         with pytest.raises(na.NovaAttnError) as ei:
             na.nova_attn_bwd_work_list(*args)
         assert ei.value.status == na.ERR_SHAPE
+
+
+def test_random_shapes_cover_every_item_once():
+    """Seeded random problems, including ones with many small heads and with more CTAs than items."""
+    import random
+    rng = random.Random(7)
+    for _ in range(40):
+        BH = rng.choice([1, 2, 5, 17, 96, 200, 777, 3000])
+        T = rng.choice([1, 127, 128, 129, 640, 1500, 4096, 20000])
+        D = rng.choice([64, 128])
+        causal = rng.random() < 0.7
+        n_ctas = rng.choice([1, 3, 64, 148, 160])
+        n_tiles = (T + 127) // 128
+        if BH * n_tiles > 40000:
+            continue
+        seen = set()
+        loads = []
+        for cta in range(n_ctas):
+            items, (chunk, n_chunks, _, _) = na.nova_attn_bwd_work_list(BH, T, D, causal, n_ctas, cta)
+            assert 1 <= chunk <= BH and n_chunks == -(-BH // chunk)
+            for it in items:
+                assert it not in seen
+                seen.add(it)
+            loads.append(sum((n_tiles - kt) if causal else n_tiles for kt, _ in items))
+        assert len(seen) == BH * n_tiles, (BH, T, D, causal, n_ctas)
+        assert all(0 <= kt < n_tiles and 0 <= bh < BH for kt, bh in seen)
+        grid = min(n_ctas, BH * n_tiles)
+        mean = sum(loads) / grid
+        # no CTA carries more than the mean plus one heaviest item and a tenth
+        assert max(loads) <= mean * 1.1 + n_tiles, (BH, T, D, causal, n_ctas, max(loads), mean)
